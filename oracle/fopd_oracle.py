@@ -1,0 +1,212 @@
+"""ctypes front end of the fp64 CPU oracle (``fopd_oracle.c``).
+
+TEST INFRASTRUCTURE, NOT PRODUCT CODE.  Only the tests, the smoke check and the
+benchmark's CPU-baseline leg may import this module; the CUDA library and its
+binding never do, and this module imports nothing from them.
+
+The functions mirror the C entry points one to one and add ``run_batch``, which
+strings them together in the order of Algorithm 1: per-token statistics for every
+chunk, per-sample sums, freshness and gate, then the objective of Eq. 16.
+Logits are numpy arrays of dtype ``float32`` or ``uint16`` (bf16 bit patterns);
+torch CPU tensors are accepted and reinterpreted without a copy.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "fopd_oracle.c")
+_LIB = os.path.join(_HERE, "libfopd_oracle.so")
+
+BF16, F32 = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (no fast-math, OpenMP over rows)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(
+            ["gcc", "-O2", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", _LIB, _SRC, "-lm"]
+        )
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.oracle_loss.restype = ctypes.c_double
+        _lib.oracle_num_threads.restype = ctypes.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().oracle_num_threads())
+
+
+def set_threads(n: int) -> None:
+    lib().oracle_set_threads(ctypes.c_int(int(n)))
+
+
+def _logits(a):
+    """numpy view + dtype code of a logits array (torch CPU tensor or numpy)."""
+    if hasattr(a, "detach"):  # torch tensor
+        import torch
+
+        a = a.detach().cpu().contiguous()
+        if a.dtype == torch.bfloat16:
+            a = a.view(torch.int16).numpy().view(np.uint16)
+        elif a.dtype == torch.float32:
+            a = a.numpy()
+        else:
+            raise TypeError(f"logits must be bf16 or fp32, got {a.dtype}")
+    if a.dtype == np.uint16:
+        return np.ascontiguousarray(a), BF16
+    if a.dtype == np.float32:
+        return np.ascontiguousarray(a), F32
+    raise TypeError(f"logits must be uint16 (bf16 bits) or float32, got {a.dtype}")
+
+
+def _np(a, dtype):
+    if hasattr(a, "detach"):
+        a = a.detach().cpu().numpy()
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def _p(a):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+@dataclass
+class TokenStats:
+    lse_s: np.ndarray
+    lse_t: np.ndarray
+    lp_s: np.ndarray
+    lp_t: np.ndarray
+    kl: np.ndarray
+    d: np.ndarray
+    rho: np.ndarray
+    k3: np.ndarray
+    valid: np.ndarray
+
+
+def token_stats(student, teacher, tokens, behav_logprob, mask, sample_id, B) -> TokenStats:
+    """Per-token quantities of one chunk (softmax normalisers, gathered
+    log-probs, reverse-KL token loss of Eq. 12, ratio and drift integrand of
+    Eq. 10)."""
+    S, dt = _logits(student)
+    T, dt2 = _logits(teacher)
+    assert dt == dt2 and S.shape == T.shape and S.ndim == 2
+    n, V = S.shape
+    y = _np(tokens, np.int32)
+    b = _np(behav_logprob, np.float32)
+    mk = _np(mask, np.uint8)
+    sid = _np(sample_id, np.int32)
+    outs = [np.zeros(n, dtype=np.float64) for _ in range(8)]
+    valid = np.zeros(n, dtype=np.uint8)
+    lib().oracle_token_stats(
+        _p(S), _p(T), ctypes.c_int(dt), ctypes.c_int64(n), ctypes.c_int64(V), ctypes.c_int64(V),
+        _p(y), _p(b), _p(mk), _p(sid), ctypes.c_int32(B), *[_p(o) for o in outs], _p(valid),
+    )
+    return TokenStats(*outs, valid)
+
+
+def sample_accumulate(acc, sample_id, stats: TokenStats) -> None:
+    """acc[B,3] += {count, sum k3, sum kl} over the aligned rows of a chunk."""
+    sid = _np(sample_id, np.int32)
+    assert acc.dtype == np.float64 and acc.flags.c_contiguous and acc.shape[1] == 3
+    lib().oracle_sample_accumulate(
+        ctypes.c_int64(len(sid)), ctypes.c_int32(acc.shape[0]), _p(sid), _p(stats.valid),
+        _p(stats.kl), _p(stats.k3), _p(acc),
+    )
+
+
+@dataclass
+class Freshness:
+    f: np.ndarray
+    w: np.ndarray
+    D_roll: np.ndarray
+    ell: np.ndarray
+    m: np.ndarray
+    coef: np.ndarray
+    valid: np.ndarray
+
+
+def sample_freshness(acc, tau, H, d_sup, alpha, beta, xi) -> Freshness:
+    """Eq. 11 freshness, Eq. 13 ReLU gate, alignment ratio and token weight."""
+    B = acc.shape[0]
+    tau = _np(tau, np.int32)
+    H = _np(H, np.int32)
+    ds = None if d_sup is None else _np(d_sup, np.float32)
+    outs = [np.zeros(B, dtype=np.float64) for _ in range(6)]
+    valid = np.zeros(B, dtype=np.uint8)
+    lib().oracle_sample_freshness(
+        ctypes.c_int32(B), _p(np.ascontiguousarray(acc)), _p(tau), _p(H),
+        _p(ds) if ds is not None else None,
+        ctypes.c_double(alpha), ctypes.c_double(beta), ctypes.c_double(xi),
+        *[_p(o) for o in outs], _p(valid),
+    )
+    return Freshness(*outs, valid)
+
+
+def loss(fr: Freshness, lam):
+    """Eq. 16 / Algorithm 1: (1/B) sum_i w_i (l_i + lambda D_roll_i)."""
+    per = np.zeros(len(fr.w), dtype=np.float64)
+    total = lib().oracle_loss(
+        ctypes.c_int32(len(fr.w)), _p(fr.w), _p(fr.ell), _p(fr.D_roll), ctypes.c_double(lam), _p(per)
+    )
+    return float(total), per
+
+
+def grad_rows(student, teacher, tokens, behav_logprob, mask, sample_id, coef, lam, rows):
+    """d L / d student logits for the listed rows, [len(rows), V] float64."""
+    S, dt = _logits(student)
+    T, dt2 = _logits(teacher)
+    assert dt == dt2 and S.shape == T.shape
+    n, V = S.shape
+    y = _np(tokens, np.int32)
+    b = _np(behav_logprob, np.float32)
+    mk = _np(mask, np.uint8)
+    sid = _np(sample_id, np.int32)
+    coef = _np(coef, np.float64)
+    rows = _np(rows, np.int64)
+    assert rows.size == 0 or (rows.min() >= 0 and rows.max() < n)
+    out = np.zeros((len(rows), V), dtype=np.float64)
+    lib().oracle_grad_rows(
+        _p(S), _p(T), ctypes.c_int(dt), ctypes.c_int64(V), ctypes.c_int64(V), _p(y), _p(b), _p(mk),
+        _p(sid), ctypes.c_int32(len(coef)), _p(coef), ctypes.c_double(lam), _p(rows),
+        ctypes.c_int64(len(rows)), _p(out),
+    )
+    return out
+
+
+@dataclass
+class BatchResult:
+    stats: list  # TokenStats per chunk
+    acc: np.ndarray  # [B,3]
+    fresh: Freshness
+    loss: float
+    per_sample_loss: np.ndarray
+
+
+def run_batch(chunks, B, tau, H, d_sup, alpha, beta, xi, lam) -> BatchResult:
+    """Algorithm 1's measurement phase then its minibatch objective, over a
+    batch supplied as a list of chunks.  Each chunk is a dict with keys
+    student, teacher, tokens, behav_logprob, mask, sample_id."""
+    acc = np.zeros((B, 3), dtype=np.float64)
+    stats = []
+    for c in chunks:
+        st = token_stats(c["student"], c["teacher"], c["tokens"], c["behav_logprob"],
+                         c["mask"], c["sample_id"], B)
+        sample_accumulate(acc, c["sample_id"], st)
+        stats.append(st)
+    fr = sample_freshness(acc, tau, H, d_sup, alpha, beta, xi)
+    total, per = loss(fr, lam)
+    return BatchResult(stats, acc, fr, total, per)
