@@ -1,0 +1,208 @@
+/*
+ * libfopd -- fused loss path of freshness-aware on-policy distillation (f-OPD)
+ * for NVIDIA B200 (sm_100a).  C ABI: plain pointers and sizes, no C++ or
+ * framework types.
+ *
+ * What the path computes (citations are to the f-OPD paper):
+ *
+ *   per token row n (student logits S[n,:], teacher logits T[n,:], stored token
+ *   y_n, behaviour log-prob b_n = log pi^{r(i)}(y_n), loss mask):
+ *     lse_s, lse_t   log-normalisers of the softmax policies          (Sec. 3.1)
+ *     lp_s, lp_t     log-probabilities of y_n under student / teacher  (Sec. 4.1)
+ *     kl_n           token loss of Eq. 12, read as the full-vocabulary reverse
+ *                    KL  sum_v p_s(v) (log p_s(v) - log p_t(v))
+ *     rho_n, k3_n    policy ratio exp(lp_s - b_n) and the per-token integrand
+ *                    rho log rho - rho + 1 of the rollout drift D_roll (Eq. 10)
+ *   per sample i (rows with mask = 1 are its aligned positions U_i):
+ *     D_roll_i, l_i  means of k3_n and kl_n over U_i                (Eq. 10, 12)
+ *     f_i            exp(-alpha sqrt(D_roll_i) - beta sqrt(D_sup_i)) / (tau_i+1)
+ *                                                                      (Eq. 11)
+ *     w_i            max(f_i - xi, 0), the ReLU gate                   (Eq. 13)
+ *     m_i            |U_i| / H_i, the alignment ratio             (Algorithm 1)
+ *   per batch:
+ *     L = (1/B) sum_i w_i (l_i + lambda D_roll_i)          (Eq. 16, Algorithm 1)
+ *     dL/dS[n,v] with w_i held constant.
+ *
+ * Calling sequence for one batch of B samples supplied in one or more chunks of
+ * token rows (rows of a sample are contiguous, in order, within and across
+ * chunks):
+ *
+ *     zero acc[B,4], loss_acc[B,2], status[1]
+ *     for each chunk:  fopd_token_stats(...)      measurement phase of Algorithm 1
+ *     fopd_sample_freshness(...)                  Eq. 11, Eq. 13
+ *     for each chunk:  fopd_loss_fwd_bwd(...)     Eq. 16 and its gradient
+ *     fopd_loss_finalize(...)
+ *     fopd_check_status(...)
+ *
+ * Memory and ownership.  Unless a parameter says HOST, every pointer is a DEVICE
+ * pointer to memory the caller owns; the library keeps no pointer after a call
+ * returns and has no global state.  Where a call needs temporary device memory
+ * that the caller did not supply (see row_ws) it takes it from the CUDA
+ * stream-ordered allocator on the caller's stream and returns it there.  All
+ * work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default
+ * stream) and the call returns without synchronising, except
+ * fopd_check_status.
+ *
+ * Errors.  Every function returns FOPD_OK or a negative fopd_status found on
+ * the host before anything is enqueued.  Conditions only visible on the device
+ * (a token or sample id out of range, tau < 0, H <= 0) never trap: the kernel
+ * ORs a bit into *status (if status is not NULL), treats the row as masked or
+ * the sample as invalid, and carries on.
+ */
+#ifndef FOPD_H_
+#define FOPD_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FOPD_VERSION 100
+
+typedef enum { FOPD_BF16 = 0, FOPD_F32 = 1 } fopd_dtype;
+
+typedef enum {
+  FOPD_OK = 0,
+  FOPD_ERR_NULL = -1,   /* a required pointer is NULL                          */
+  FOPD_ERR_ALIGN = -2,  /* logits base or row pitch not 16-byte aligned         */
+  FOPD_ERR_SIZE = -3,   /* negative size, row_stride < vocab, vocab too large   */
+  FOPD_ERR_DTYPE = -4,  /* dtype is neither FOPD_BF16 nor FOPD_F32              */
+  FOPD_ERR_PARAM = -5,  /* alpha/beta negative or a parameter not finite        */
+  FOPD_ERR_CUDA = -6,   /* a CUDA runtime call failed (launch, allocation)      */
+  FOPD_ERR_ALIAS = -7,  /* dlogits overlaps student or teacher                  */
+  FOPD_ERR_DEVICE = -8  /* fopd_check_status: the device status word is non-zero */
+} fopd_status;
+
+/* Bits ORed into the device status word. */
+#define FOPD_DEV_BAD_TOKEN 1    /* mask = 1 row with token outside [0, vocab)   */
+#define FOPD_DEV_BAD_SAMPLE 2   /* row with sample id outside [0, B)            */
+#define FOPD_DEV_BAD_TAU 4      /* staleness < 0                                */
+#define FOPD_DEV_BAD_LENGTH 8   /* seq_len <= 0 or aligned count > seq_len      */
+
+/* alpha, beta >= 0 scale the two drift diagnostics (Eq. 11); xi is the gate
+ * threshold (Eq. 13); lambda weights the rollout anchor (Eq. 16).  The paper
+ * gives no values; they are run-time parameters. */
+typedef struct {
+  float alpha, beta, xi, lambda;
+} fopd_params;
+
+/* One chunk of token rows.  student/teacher: [n_rows, vocab] row-major with a
+ * pitch of row_stride elements (row_stride >= vocab), same dtype; base address
+ * and pitch in bytes must be multiples of 16.  Rows with mask = 0 (padding,
+ * tool output) are never read. */
+typedef struct {
+  const void *student;
+  const void *teacher;
+  const float *behav_logprob; /* [n_rows] log pi_behaviour(y_n)                 */
+  const int32_t *tokens;      /* [n_rows] 0 <= y_n < vocab                      */
+  const uint8_t *mask;        /* [n_rows] 1 = aligned response token            */
+  const int32_t *sample_id;   /* [n_rows] 0 <= id < B, non-decreasing           */
+  int64_t n_rows;
+  int64_t vocab;
+  int64_t row_stride;
+  int32_t dtype;              /* fopd_dtype                                     */
+} fopd_chunk;
+
+/* Columns of the per-row workspace row_ws[n_rows, 4] (fp32). */
+#define FOPD_WS_LSE_S 0
+#define FOPD_WS_LSE_T 1
+#define FOPD_WS_KL 2
+#define FOPD_WS_D 3 /* d_n = lp_s - b_n = log rho_n */
+
+/* Columns of acc[B, 4] (fp64): aligned-row count, sum of k3, sum of kl, rows seen. */
+#define FOPD_ACC_CNT 0
+#define FOPD_ACC_K3 1
+#define FOPD_ACC_KL 2
+#define FOPD_ACC_ROWS 3
+
+/*
+ * Per-token statistics of one chunk and their per-sample sums: one streaming
+ * pass over the student and teacher rows (online max / sum-exp), the gather of
+ * the stored token, the Eq. 12 token loss and the Eq. 10 drift integrand.
+ *
+ *   lp_s, lp_t, kl, ratio  [n_rows] fp32 outputs, any may be NULL.  Rows with
+ *                          mask = 0 or a bad id get exactly 0.
+ *   row_ws                 optional [n_rows, 4] fp32 output (columns above),
+ *                          16-byte aligned; pass it to fopd_loss_fwd_bwd for
+ *                          the same chunk to let that call skip its own
+ *                          reduction sweep.  NULL: a temporary of the same size
+ *                          is taken from the stream-ordered allocator.
+ *   acc                    [B, 4] fp64, ADDED to (the caller zeroes it before
+ *                          the first chunk of a batch).  The sums are formed in
+ *                          a fixed order, so results are reproducible bit for bit.
+ *   status                 device int32 status word, or NULL.
+ */
+int fopd_token_stats(const fopd_chunk *chunk /* HOST */, int32_t B, float *lp_s,
+                     float *lp_t, float *kl, float *ratio, float *row_ws,
+                     double *acc, int32_t *status, void *stream);
+
+/*
+ * Per-sample freshness (Eq. 11), ReLU gate (Eq. 13), alignment ratio and the
+ * per-token weight coef_i = w_i / (B |U_i|) that fopd_loss_fwd_bwd applies.
+ * A sample with no aligned row, seq_len <= 0 or staleness < 0 is invalid:
+ * f = w = m = coef = 0 (Algorithm 1, the |U| = 0 branch).
+ *
+ *   acc        [B, 4] fp64 from fopd_token_stats (all chunks done)
+ *   staleness  [B] int32 tau_i = t - r(i);  seq_len [B] int32 H_i
+ *   d_sup      [B] fp32 supervision drift D_sup_i, or NULL for 0 (teacher and
+ *              context unchanged since grading)
+ *   f, w, d_roll, l_distill, m_align, coef   [B] fp32 outputs; coef is
+ *              required, the others may be NULL
+ *   buffer_means  optional [2] fp32: mean f_i and mean m_i over the B samples
+ *              (the buffer statistics of Eq. 14)
+ */
+int fopd_sample_freshness(const double *acc, const int32_t *staleness,
+                          const int32_t *seq_len, const float *d_sup, int32_t B,
+                          fopd_params p, float *f, float *w, float *d_roll,
+                          float *l_distill, float *m_align, float *coef,
+                          float *buffer_means, int32_t *status, void *stream);
+
+/*
+ * Fused loss forward + backward for one chunk (Eq. 16 with w_i constant).  For
+ * an aligned row n of a sample with coef_i != 0:
+ *
+ *   dlogits[n,v] = coef_i { p_s(v) [ (log p_s(v) - log p_t(v)) - kl_n ]
+ *                           + lambda rho_n d_n ( 1[v = y_n] - p_s(v) ) }
+ *
+ * Every other row of dlogits (masked, padded, bad id, gated or invalid sample)
+ * is written as +0 and its logits are not read.  The per-sample sums of kl and
+ * k3 over the rows this call differentiated are ADDED to loss_acc.
+ *
+ *   coef      [B] fp32 from fopd_sample_freshness
+ *   row_ws    the workspace fopd_token_stats wrote for THIS chunk, or NULL.
+ *             With it the call is one streaming pass (read S, read T, write
+ *             dlogits).  Without it the kernel stages each row on chip, does
+ *             the reduction sweep and the gradient sweep from there, and still
+ *             reads S and T from memory once.
+ *   dlogits   [n_rows, vocab] with the same dtype and pitch as student; must
+ *             not overlap student or teacher
+ *   loss_acc  [B, 2] fp64 {sum kl, sum k3}, ADDED to; caller zeroes per batch
+ */
+int fopd_loss_fwd_bwd(const fopd_chunk *chunk /* HOST */, int32_t B,
+                      const float *coef, const float *row_ws, fopd_params p,
+                      void *dlogits, double *loss_acc, int32_t *status,
+                      void *stream);
+
+/*
+ * After the last chunk: per_sample_loss[i] = w_i (l_i + lambda D_roll_i) with
+ * l_i, D_roll_i = loss_acc[i] / acc[i].cnt, and loss_out[0] = (1/B) sum_i of
+ * it (Eq. 16; Algorithm 1 divides by the minibatch size, gated samples
+ * included).  per_sample_loss may be NULL.
+ */
+int fopd_loss_finalize(const double *loss_acc, const double *acc, const float *w,
+                       int32_t B, fopd_params p, float *per_sample_loss,
+                       float *loss_out, void *stream);
+
+/* Synchronises `stream`, reads the device status word and returns FOPD_OK,
+ * FOPD_ERR_DEVICE (word non-zero; *bits_out receives it if not NULL, HOST) or
+ * FOPD_ERR_CUDA. */
+int fopd_check_status(const int32_t *status, int32_t *bits_out /* HOST */, void *stream);
+
+const char *fopd_strerror(int code);
+int fopd_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FOPD_H_ */

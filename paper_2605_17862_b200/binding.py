@@ -1,0 +1,165 @@
+"""Thin ctypes binding of libfopd.so: same names as the C ABI, torch tensors in,
+pointers out.  Argument marshalling only -- every step of the path runs in the
+library's CUDA kernels.  There is no CPU fallback: if the shared library is
+missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfopd.so")
+
+FOPD_BF16, FOPD_F32 = 0, 1
+
+EXPORTS = (
+    "fopd_token_stats", "fopd_sample_freshness", "fopd_loss_fwd_bwd", "fopd_loss_finalize",
+    "fopd_check_status", "fopd_strerror", "fopd_version",
+)
+
+
+class FopdError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} (status {code})")
+
+
+class fopd_params(ctypes.Structure):
+    _fields_ = [("alpha", ctypes.c_float), ("beta", ctypes.c_float), ("xi", ctypes.c_float),
+                ("lam", ctypes.c_float)]
+
+
+class fopd_chunk(ctypes.Structure):
+    _fields_ = [
+        ("student", ctypes.c_void_p), ("teacher", ctypes.c_void_p), ("behav_logprob", ctypes.c_void_p),
+        ("tokens", ctypes.c_void_p), ("mask", ctypes.c_void_p), ("sample_id", ctypes.c_void_p),
+        ("n_rows", ctypes.c_int64), ("vocab", ctypes.c_int64), ("row_stride", ctypes.c_int64),
+        ("dtype", ctypes.c_int32),
+    ]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libfopd.so (built in-tree by ``build.build_lib``); fails loudly if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} not found: build it with `python -m paper_2605_17862_b200.build` "
+                "(there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32 = ctypes.c_void_p, ctypes.c_int32
+        L.fopd_version.restype = ctypes.c_int
+        L.fopd_strerror.restype = ctypes.c_char_p
+        L.fopd_strerror.argtypes = [ctypes.c_int]
+        L.fopd_token_stats.argtypes = [ctypes.POINTER(fopd_chunk), i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.fopd_sample_freshness.argtypes = [vp, vp, vp, vp, i32, fopd_params, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.fopd_loss_fwd_bwd.argtypes = [ctypes.POINTER(fopd_chunk), i32, vp, vp, fopd_params, vp, vp, vp, vp]
+        L.fopd_loss_finalize.argtypes = [vp, vp, vp, i32, fopd_params, vp, vp, vp]
+        L.fopd_check_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
+        for name in EXPORTS:
+            getattr(L, name)
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().fopd_strerror(int(code)).decode()
+
+
+def version() -> int:
+    return int(lib().fopd_version())
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check(rc: int, where: str):
+    if rc != 0:
+        raise FopdError(rc, where)
+
+
+def params(alpha=1.0, beta=1.0, xi=0.15, lam=0.1) -> fopd_params:
+    return fopd_params(float(alpha), float(beta), float(xi), float(lam))
+
+
+@dataclass
+class Chunk:
+    """Device tensors of one chunk of token rows (see ``fopd_chunk`` in fopd.h)."""
+    student: torch.Tensor  # [n, V] (row pitch = student.stride(0)), bf16 or fp32
+    teacher: torch.Tensor
+    behav_logprob: torch.Tensor  # [n] fp32
+    tokens: torch.Tensor  # [n] int32
+    mask: torch.Tensor  # [n] uint8
+    sample_id: torch.Tensor  # [n] int32
+    vocab: int | None = None  # columns in use; defaults to student.shape[1]
+
+    def c_struct(self) -> fopd_chunk:
+        S, T = self.student, self.teacher
+        assert S.dtype == T.dtype and S.dtype in (torch.bfloat16, torch.float32)
+        assert S.dim() == 2 and S.shape == T.shape and S.stride() == T.stride() and S.stride(1) == 1
+        assert self.behav_logprob.dtype == torch.float32 and self.tokens.dtype == torch.int32
+        assert self.mask.dtype == torch.uint8 and self.sample_id.dtype == torch.int32
+        n = S.shape[0]
+        for t in (self.behav_logprob, self.tokens, self.mask, self.sample_id):
+            assert t.is_contiguous() and t.numel() == n and t.device == S.device
+        return fopd_chunk(
+            S.data_ptr(), T.data_ptr(), self.behav_logprob.data_ptr(), self.tokens.data_ptr(),
+            self.mask.data_ptr(), self.sample_id.data_ptr(), n, self.vocab or S.shape[1],
+            S.stride(0) if n > 1 else max(S.stride(0), S.shape[1]),
+            FOPD_BF16 if S.dtype == torch.bfloat16 else FOPD_F32,
+        )
+
+
+def fopd_token_stats(chunk: Chunk, B: int, acc, *, lp_s=None, lp_t=None, kl=None, ratio=None,
+                     row_ws=None, status=None, stream=None):
+    c = chunk.c_struct()
+    _check(lib().fopd_token_stats(ctypes.byref(c), B, _ptr(lp_s), _ptr(lp_t), _ptr(kl), _ptr(ratio),
+                                  _ptr(row_ws), _ptr(acc), _ptr(status), _stream(stream)),
+           "fopd_token_stats")
+
+
+def fopd_sample_freshness(acc, staleness, seq_len, d_sup, B: int, p: fopd_params, *, coef, f=None,
+                          w=None, d_roll=None, l_distill=None, m_align=None, buffer_means=None,
+                          status=None, stream=None):
+    _check(lib().fopd_sample_freshness(_ptr(acc), _ptr(staleness), _ptr(seq_len), _ptr(d_sup), B, p,
+                                       _ptr(f), _ptr(w), _ptr(d_roll), _ptr(l_distill), _ptr(m_align),
+                                       _ptr(coef), _ptr(buffer_means), _ptr(status), _stream(stream)),
+           "fopd_sample_freshness")
+
+
+def fopd_loss_fwd_bwd(chunk: Chunk, B: int, coef, p: fopd_params, dlogits, loss_acc, *, row_ws=None,
+                      status=None, stream=None):
+    c = chunk.c_struct()
+    assert dlogits.dtype == chunk.student.dtype and dlogits.stride() == chunk.student.stride()
+    _check(lib().fopd_loss_fwd_bwd(ctypes.byref(c), B, _ptr(coef), _ptr(row_ws), p, _ptr(dlogits),
+                                   _ptr(loss_acc), _ptr(status), _stream(stream)),
+           "fopd_loss_fwd_bwd")
+
+
+def fopd_loss_finalize(loss_acc, acc, w, B: int, p: fopd_params, loss_out, *, per_sample_loss=None,
+                       stream=None):
+    _check(lib().fopd_loss_finalize(_ptr(loss_acc), _ptr(acc), _ptr(w), B, p, _ptr(per_sample_loss),
+                                    _ptr(loss_out), _stream(stream)),
+           "fopd_loss_finalize")
+
+
+def fopd_check_status(status, stream=None) -> int:
+    """Synchronises the stream and returns the device status bits (0 = clean)."""
+    bits = ctypes.c_int32(0)
+    rc = lib().fopd_check_status(_ptr(status), ctypes.byref(bits), _stream(stream))
+    if rc not in (0, -8):
+        raise FopdError(rc, "fopd_check_status")
+    return int(bits.value)

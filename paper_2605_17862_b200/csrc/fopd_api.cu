@@ -1,0 +1,208 @@
+// C ABI of libfopd: argument checks on the host, kernel launches on the
+// caller's stream.  See include/fopd.h for the contract of every entry point.
+#include <cmath>
+#include <cstdio>
+
+#include "stream_kernels.cuh"
+
+using namespace fopd;
+
+namespace {
+
+struct DeviceInfo {
+  int sm_count = 0;
+};
+
+int device_info(DeviceInfo *out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FOPD_ERR_CUDA;
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return FOPD_ERR_CUDA;
+  out->sm_count = sms;
+  return FOPD_OK;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_chunk(const fopd_chunk *c, int32_t B) {
+  if (!c) return FOPD_ERR_NULL;
+  if (c->dtype != FOPD_BF16 && c->dtype != FOPD_F32) return FOPD_ERR_DTYPE;
+  if (c->n_rows < 0 || c->vocab <= 0 || c->row_stride < c->vocab || B <= 0) return FOPD_ERR_SIZE;
+  if (c->vocab > (int64_t)1 << 30 || c->n_rows > (int64_t)1 << 40) return FOPD_ERR_SIZE;
+  if (c->n_rows == 0) return FOPD_OK;
+  if (!c->student || !c->teacher || !c->behav_logprob || !c->tokens || !c->mask || !c->sample_id)
+    return FOPD_ERR_NULL;
+  const int64_t esz = c->dtype == FOPD_BF16 ? 2 : 4;
+  if (!aligned16(c->student) || !aligned16(c->teacher) || (c->row_stride * esz) % 16 != 0)
+    return FOPD_ERR_ALIGN;
+  return FOPD_OK;
+}
+
+ChunkDev to_dev(const fopd_chunk *c) {
+  ChunkDev d;
+  d.student = c->student;
+  d.teacher = c->teacher;
+  d.behav = c->behav_logprob;
+  d.tokens = c->tokens;
+  d.mask = c->mask;
+  d.sid = c->sample_id;
+  d.n_rows = c->n_rows;
+  d.vocab = c->vocab;
+  d.stride = c->row_stride;
+  return d;
+}
+
+int check_params(const fopd_params &p) {
+  if (!std::isfinite(p.alpha) || !std::isfinite(p.beta) || !std::isfinite(p.xi) || !std::isfinite(p.lambda))
+    return FOPD_ERR_PARAM;
+  if (p.alpha < 0.f || p.beta < 0.f) return FOPD_ERR_PARAM;
+  return FOPD_OK;
+}
+
+int launch_ok() { return cudaGetLastError() == cudaSuccess ? FOPD_OK : FOPD_ERR_CUDA; }
+
+int stream_grid(const DeviceInfo &di, int64_t n_rows) {
+  const int64_t persistent = (int64_t)di.sm_count * 2;  // two 512-thread CTAs per SM
+  return (int)(n_rows < persistent ? n_rows : persistent);
+}
+
+// Enqueues the statistics sweep of a chunk into row_ws (and the optional
+// per-row outputs).
+int launch_stats(const fopd_chunk *c, int32_t B, float *lp_s, float *lp_t, float *kl, float *ratio,
+                 float *row_ws, int32_t *status, cudaStream_t st, const DeviceInfo &di) {
+  const ChunkDev d = to_dev(c);
+  const int grid = stream_grid(di, c->n_rows);
+  if (c->dtype == FOPD_BF16)
+    token_stats_kernel<FOPD_BF16><<<grid, kStreamThreads, 0, st>>>(d, B, lp_s, lp_t, kl, ratio, row_ws, status);
+  else
+    token_stats_kernel<FOPD_F32><<<grid, kStreamThreads, 0, st>>>(d, B, lp_s, lp_t, kl, ratio, row_ws, status);
+  return launch_ok();
+}
+
+}  // namespace
+
+extern "C" {
+
+int fopd_version(void) { return FOPD_VERSION; }
+
+const char *fopd_strerror(int code) {
+  switch (code) {
+    case FOPD_OK: return "ok";
+    case FOPD_ERR_NULL: return "a required pointer is NULL";
+    case FOPD_ERR_ALIGN: return "logits base, row pitch or workspace not 16-byte aligned";
+    case FOPD_ERR_SIZE: return "bad size (negative, row_stride < vocab, or too large)";
+    case FOPD_ERR_DTYPE: return "dtype must be FOPD_BF16 or FOPD_F32";
+    case FOPD_ERR_PARAM: return "alpha/beta must be >= 0 and all parameters finite";
+    case FOPD_ERR_CUDA: return "a CUDA runtime call failed";
+    case FOPD_ERR_ALIAS: return "dlogits overlaps student or teacher";
+    case FOPD_ERR_DEVICE: return "device status word is non-zero (bad token/sample id, staleness or length)";
+    default: return "unknown fopd status";
+  }
+}
+
+int fopd_token_stats(const fopd_chunk *chunk, int32_t B, float *lp_s, float *lp_t, float *kl,
+                     float *ratio, float *row_ws, double *acc, int32_t *status, void *stream) {
+  int rc = check_chunk(chunk, B);
+  if (rc != FOPD_OK) return rc;
+  if (!acc) return FOPD_ERR_NULL;
+  if (row_ws && !aligned16(row_ws)) return FOPD_ERR_ALIGN;
+  if (chunk->n_rows == 0) return FOPD_OK;
+  DeviceInfo di;
+  if ((rc = device_info(&di)) != FOPD_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  float *ws = row_ws;
+  if (!ws) {
+    if (cudaMallocAsync(reinterpret_cast<void **>(&ws), (size_t)chunk->n_rows * 4 * sizeof(float), st) !=
+        cudaSuccess)
+      return FOPD_ERR_CUDA;
+  }
+  rc = launch_stats(chunk, B, lp_s, lp_t, kl, ratio, ws, status, st, di);
+  if (rc == FOPD_OK) {
+    segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(to_dev(chunk), B, ws, nullptr, 0, acc);
+    rc = launch_ok();
+  }
+  if (!row_ws && cudaFreeAsync(ws, st) != cudaSuccess) rc = FOPD_ERR_CUDA;
+  return rc;
+}
+
+int fopd_sample_freshness(const double *acc, const int32_t *staleness, const int32_t *seq_len,
+                          const float *d_sup, int32_t B, fopd_params p, float *f, float *w,
+                          float *d_roll, float *l_distill, float *m_align, float *coef,
+                          float *buffer_means, int32_t *status, void *stream) {
+  if (B <= 0) return FOPD_ERR_SIZE;
+  if (!acc || !staleness || !seq_len || !coef) return FOPD_ERR_NULL;
+  int rc = check_params(p);
+  if (rc != FOPD_OK) return rc;
+  freshness_kernel<<<1, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+      acc, staleness, seq_len, d_sup, B, p, f, w, d_roll, l_distill, m_align, coef, buffer_means, status);
+  return launch_ok();
+}
+
+int fopd_loss_fwd_bwd(const fopd_chunk *chunk, int32_t B, const float *coef, const float *row_ws,
+                      fopd_params p, void *dlogits, double *loss_acc, int32_t *status, void *stream) {
+  int rc = check_chunk(chunk, B);
+  if (rc != FOPD_OK) return rc;
+  if ((rc = check_params(p)) != FOPD_OK) return rc;
+  if (!coef || !loss_acc) return FOPD_ERR_NULL;
+  if (chunk->n_rows == 0) return FOPD_OK;
+  if (!dlogits) return FOPD_ERR_NULL;
+  if (!aligned16(dlogits) || (row_ws && !aligned16(row_ws))) return FOPD_ERR_ALIGN;
+  {
+    const int64_t esz = chunk->dtype == FOPD_BF16 ? 2 : 4;
+    const uintptr_t bytes = (uintptr_t)(chunk->n_rows * chunk->row_stride * esz);
+    const uintptr_t o = (uintptr_t)dlogits, s = (uintptr_t)chunk->student, t = (uintptr_t)chunk->teacher;
+    if ((o < s + bytes && s < o + bytes) || (o < t + bytes && t < o + bytes)) return FOPD_ERR_ALIAS;
+  }
+  DeviceInfo di;
+  if ((rc = device_info(&di)) != FOPD_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const ChunkDev d = to_dev(chunk);
+  const float *ws = row_ws;
+  float *tmp = nullptr;
+  if (!ws) {
+    // No cached statistics: redo the reduction sweep into a temporary workspace.
+    if (cudaMallocAsync(reinterpret_cast<void **>(&tmp), (size_t)chunk->n_rows * 4 * sizeof(float), st) !=
+        cudaSuccess)
+      return FOPD_ERR_CUDA;
+    rc = launch_stats(chunk, B, nullptr, nullptr, nullptr, nullptr, tmp, status, st, di);
+    ws = tmp;
+  }
+  if (rc == FOPD_OK) {
+    const int grid = stream_grid(di, chunk->n_rows);
+    if (chunk->dtype == FOPD_BF16)
+      grad_stream_kernel<FOPD_BF16><<<grid, kStreamThreads, 0, st>>>(d, B, coef, ws, p.lambda, dlogits);
+    else
+      grad_stream_kernel<FOPD_F32><<<grid, kStreamThreads, 0, st>>>(d, B, coef, ws, p.lambda, dlogits);
+    rc = launch_ok();
+  }
+  if (rc == FOPD_OK) {
+    segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(d, B, ws, coef, 1, loss_acc);
+    rc = launch_ok();
+  }
+  if (tmp && cudaFreeAsync(tmp, st) != cudaSuccess) rc = FOPD_ERR_CUDA;
+  return rc;
+}
+
+int fopd_loss_finalize(const double *loss_acc, const double *acc, const float *w, int32_t B,
+                       fopd_params p, float *per_sample_loss, float *loss_out, void *stream) {
+  if (B <= 0) return FOPD_ERR_SIZE;
+  if (!loss_acc || !acc || !w || !loss_out) return FOPD_ERR_NULL;
+  int rc = check_params(p);
+  if (rc != FOPD_OK) return rc;
+  finalize_kernel<<<1, 256, 0, static_cast<cudaStream_t>(stream)>>>(loss_acc, acc, w, B, p.lambda,
+                                                                    per_sample_loss, loss_out);
+  return launch_ok();
+}
+
+int fopd_check_status(const int32_t *status, int32_t *bits_out, void *stream) {
+  if (!status) return FOPD_ERR_NULL;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int32_t bits = 0;
+  if (cudaMemcpyAsync(&bits, status, sizeof(bits), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return FOPD_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return FOPD_ERR_CUDA;
+  if (bits_out) *bits_out = bits;
+  return bits == 0 ? FOPD_OK : FOPD_ERR_DEVICE;
+}
+
+}  // extern "C"

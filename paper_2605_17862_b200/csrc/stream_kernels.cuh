@@ -1,0 +1,363 @@
+// Streaming kernels of libfopd that work for any vocabulary size and both
+// logit dtypes: the statistics sweep, the single-pass gradient sweep that uses
+// cached row statistics, the per-sample segmented reduction, freshness and
+// the final loss.  One CTA walks one row at a time (persistent, row = blockIdx
+// + k * gridDim); rows are 16-byte aligned so the body uses 16-byte loads and a
+// scalar tail covers vocabularies that do not fill the last vector.
+#pragma once
+
+#include "common.cuh"
+
+namespace fopd {
+
+constexpr int kStreamThreads = 512;
+constexpr int kUnroll = 4;
+
+struct ChunkDev {
+  const void *student, *teacher;
+  const float *behav;
+  const int32_t *tokens;
+  const uint8_t *mask;
+  const int32_t *sid;
+  int64_t n_rows, vocab, stride;
+};
+
+// Is row n aligned (counts towards U_i)?  Records bad ids in the status word.
+__device__ __forceinline__ bool row_is_aligned(const ChunkDev &c, int64_t n, int32_t B,
+                                               int32_t *status, bool report) {
+  const int32_t sid = c.sid[n];
+  bool ok = true;
+  if (sid < 0 || sid >= B) {
+    if (report && status) atomicOr(status, FOPD_DEV_BAD_SAMPLE);
+    ok = false;
+  }
+  if (c.mask[n] == 0) return false;
+  const int32_t y = c.tokens[n];
+  if (y < 0 || y >= c.vocab) {
+    if (report && status) atomicOr(status, FOPD_DEV_BAD_TOKEN);
+    ok = false;
+  }
+  return ok;
+}
+
+// Turns the finished accumulators of a row into the quantities of Sec. 4.1 /
+// Eq. 10 / Eq. 12 and writes the per-row outputs.  Called by one thread.
+template <int DT>
+__device__ __forceinline__ void finish_row(const ChunkDev &c, int64_t n, const RowAcc &r, float *lp_s,
+                                           float *lp_t, float *kl_out, float *ratio, float *row_ws) {
+  using E = Elem<DT>;
+  // log of the partition sums in full precision (logf, not the fast intrinsic)
+  const float ls = r.ms + logf(r.zs);
+  const float lt = r.mt + logf(r.zt);
+  const float kl = r.as / r.zs - (ls - lt);
+  const int32_t y = c.tokens[n];
+  const float sy = E::load1(c.student, n * c.stride + y);
+  const float ty = E::load1(c.teacher, n * c.stride + y);
+  const float lps = sy - ls, lpt = ty - lt;
+  const float d = lps - c.behav[n];
+  if (lp_s) lp_s[n] = lps;
+  if (lp_t) lp_t[n] = lpt;
+  if (kl_out) kl_out[n] = kl;
+  if (ratio) ratio[n] = (float)exp((double)d);
+  reinterpret_cast<float4 *>(row_ws)[n] = make_float4(ls, lt, kl, d);
+}
+
+__device__ __forceinline__ void zero_row_outputs(int64_t n, float *lp_s, float *lp_t, float *kl_out,
+                                                 float *ratio, float *row_ws) {
+  if (lp_s) lp_s[n] = 0.f;
+  if (lp_t) lp_t[n] = 0.f;
+  if (kl_out) kl_out[n] = 0.f;
+  if (ratio) ratio[n] = 0.f;
+  reinterpret_cast<float4 *>(row_ws)[n] = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
+// Sweep one row from global memory into a per-thread RowAcc.
+template <int DT, int kThreads>
+__device__ __forceinline__ RowAcc sweep_row_global(const void *srow, const void *trow, int64_t V) {
+  using E = Elem<DT>;
+  constexpr int P = E::kPerVec;
+  RowAcc acc;
+  acc.init();
+  const int64_t nvec = V / P;
+  const uint4 *s4 = reinterpret_cast<const uint4 *>(srow);
+  const uint4 *t4 = reinterpret_cast<const uint4 *>(trow);
+  int64_t i = threadIdx.x;
+  for (; i + (kUnroll - 1) * kThreads < nvec; i += kUnroll * kThreads) {
+    uint4 a[kUnroll], b[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      a[u] = ld_stream(s4 + i + u * kThreads);
+      b[u] = ld_stream(t4 + i + u * kThreads);
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      float s[P], t[P];
+      E::unpack(a[u], s);
+      E::unpack(b[u], t);
+      acc.add<P>(s, t);
+    }
+  }
+  for (; i < nvec; i += kThreads) {
+    float s[P], t[P];
+    E::unpack(ld_stream(s4 + i), s);
+    E::unpack(ld_stream(t4 + i), t);
+    acc.add<P>(s, t);
+  }
+  const int64_t tail = nvec * P + threadIdx.x;
+  if (tail < V) acc.add1(E::load1(srow, tail), E::load1(trow, tail));
+  return acc;
+}
+
+// a1-a4: statistics sweep.  grid = any, block = kStreamThreads.
+template <int DT>
+__global__ void __launch_bounds__(kStreamThreads, 2)
+    token_stats_kernel(ChunkDev c, int32_t B, float *lp_s, float *lp_t, float *kl, float *ratio,
+                       float *row_ws, int32_t *status) {
+  using E = Elem<DT>;
+  __shared__ RowAcc scratch[kStreamThreads / 32];
+  for (int64_t n = blockIdx.x; n < c.n_rows; n += gridDim.x) {
+    const bool ok = row_is_aligned(c, n, B, status, threadIdx.x == 0);
+    if (!ok) {
+      if (threadIdx.x == 0) zero_row_outputs(n, lp_s, lp_t, kl, ratio, row_ws);
+      continue;
+    }
+    const char *srow = reinterpret_cast<const char *>(c.student) + n * c.stride * E::kBytes;
+    const char *trow = reinterpret_cast<const char *>(c.teacher) + n * c.stride * E::kBytes;
+    RowAcc acc = sweep_row_global<DT, kStreamThreads>(srow, trow, c.vocab);
+    acc = block_reduce<kStreamThreads>(acc, scratch);
+    if (threadIdx.x == 0) finish_row<DT>(c, n, acc, lp_s, lp_t, kl, ratio, row_ws);
+    __syncthreads();  // scratch is reused by the next row
+  }
+}
+
+// Per-row constants of the gradient sweep (see fopd_loss_fwd_bwd):
+//   dS_v = cp_v * ((s_v - t_v) - K) + [v == y] * cg
+//   cp_v = coef * p_s(v) = 2^(s_v*log2e + e0),  e0 = log2(coef) - lse_s*log2e
+//   K    = kl + g + (lse_s - lse_t),  g = lambda * rho * d,  cg = coef * g
+struct GradRow {
+  float e0, K, cg;
+  int32_t y;
+};
+
+__device__ __forceinline__ GradRow make_grad_row(float4 ws, float coef, float lambda, int32_t y) {
+  const float d = ws.w;
+  const float g = lambda * (float)(exp((double)d) * (double)d);
+  GradRow r;
+  r.e0 = log2f(coef) - ws.x * kLog2e;
+  r.K = ws.z + g + (ws.x - ws.y);
+  r.cg = coef * g;
+  r.y = y;
+  return r;
+}
+
+template <int DT>
+__device__ __forceinline__ uint4 grad_vec(const uint4 &sv, const uint4 &tv, const GradRow &r,
+                                          int64_t v0) {
+  using E = Elem<DT>;
+  constexpr int P = E::kPerVec;
+  float s[P], t[P], o[P];
+  E::unpack(sv, s);
+  E::unpack(tv, t);
+#pragma unroll
+  for (int i = 0; i < P; ++i) {
+    const float cp = ex2(fmaf(s[i], kLog2e, r.e0));
+    o[i] = cp * ((s[i] - t[i]) - r.K);
+  }
+  const int64_t off = (int64_t)r.y - v0;
+  if (off >= 0 && off < P) {
+#pragma unroll
+    for (int i = 0; i < P; ++i)
+      if (i == off) o[i] += r.cg;
+  }
+  return E::pack(o);
+}
+
+// a8 with cached row statistics: one streaming pass, read S, read T, write dS.
+template <int DT>
+__global__ void __launch_bounds__(kStreamThreads, 2)
+    grad_stream_kernel(ChunkDev c, int32_t B, const float *coef, const float *row_ws, float lambda,
+                       void *dlogits) {
+  using E = Elem<DT>;
+  constexpr int P = E::kPerVec;
+  constexpr int kThreads = kStreamThreads;
+  const int64_t V = c.vocab, nvec = V / P;
+  for (int64_t n = blockIdx.x; n < c.n_rows; n += gridDim.x) {
+    char *orow = reinterpret_cast<char *>(dlogits) + n * c.stride * E::kBytes;
+    uint4 *o4 = reinterpret_cast<uint4 *>(orow);
+    float cf = 0.f;
+    if (row_is_aligned(c, n, B, nullptr, false)) cf = coef[c.sid[n]];
+    if (!(cf > 0.f)) {  // masked, padded, bad id, gated or invalid sample: +0
+      const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+      for (int64_t i = threadIdx.x; i < nvec; i += kThreads) st_stream(o4 + i, z);
+      const int64_t tail = nvec * P + threadIdx.x;
+      if (tail < V) E::store1(orow, tail, 0.f);
+      continue;
+    }
+    const GradRow r = make_grad_row(reinterpret_cast<const float4 *>(row_ws)[n], cf, lambda, c.tokens[n]);
+    const char *srow = reinterpret_cast<const char *>(c.student) + n * c.stride * E::kBytes;
+    const char *trow = reinterpret_cast<const char *>(c.teacher) + n * c.stride * E::kBytes;
+    const uint4 *s4 = reinterpret_cast<const uint4 *>(srow);
+    const uint4 *t4 = reinterpret_cast<const uint4 *>(trow);
+    int64_t i = threadIdx.x;
+    for (; i + (kUnroll - 1) * kThreads < nvec; i += kUnroll * kThreads) {
+      uint4 a[kUnroll], b[kUnroll];
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) {
+        a[u] = ld_stream(s4 + i + u * kThreads);
+        b[u] = ld_stream(t4 + i + u * kThreads);
+      }
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u)
+        st_stream(o4 + i + u * kThreads, grad_vec<DT>(a[u], b[u], r, (i + u * kThreads) * P));
+    }
+    for (; i < nvec; i += kThreads)
+      st_stream(o4 + i, grad_vec<DT>(ld_stream(s4 + i), ld_stream(t4 + i), r, i * P));
+    const int64_t tail = nvec * P + threadIdx.x;
+    if (tail < V) {
+      const float s = E::load1(srow, tail), t = E::load1(trow, tail);
+      float o = ex2(fmaf(s, kLog2e, r.e0)) * ((s - t) - r.K);
+      if (tail == r.y) o += r.cg;
+      E::store1(orow, tail, o);
+    }
+  }
+}
+
+// a5: deterministic segmented reduction of per-row statistics into per-sample
+// sums.  One block per sample; the block finds its (contiguous) row range by
+// binary search in the non-decreasing sample_id array, every thread sums a
+// fixed strided subset in fp64 and a fixed tree combines them, so a rerun
+// reproduces the bits.  mode 0: acc[B,4] += {cnt, sum k3, sum kl, rows}.
+// mode 1: loss_acc[B,2] += {sum kl, sum k3} over rows of samples with coef > 0.
+constexpr int kSegThreads = 256;
+
+__device__ __forceinline__ int64_t lower_bound_sid(const int32_t *sid, int64_t n, int32_t key) {
+  int64_t lo = 0, hi = n;
+  while (lo < hi) {
+    const int64_t mid = (lo + hi) >> 1;
+    if (sid[mid] < key) lo = mid + 1;
+    else hi = mid;
+  }
+  return lo;
+}
+
+__global__ void __launch_bounds__(kSegThreads)
+    segment_reduce_kernel(ChunkDev c, int32_t B, const float *row_ws, const float *coef, int mode,
+                          double *out) {
+  __shared__ double sh[3][kSegThreads];
+  const int32_t i = blockIdx.x;
+  if (mode == 1 && !(coef[i] > 0.f)) return;
+  const int64_t lo = lower_bound_sid(c.sid, c.n_rows, i);
+  const int64_t hi = lower_bound_sid(c.sid, c.n_rows, i + 1);
+  if (lo >= hi) return;
+  double cnt = 0.0, sk3 = 0.0, skl = 0.0;
+  for (int64_t n = lo + threadIdx.x; n < hi; n += kSegThreads) {
+    if (c.sid[n] != i || c.mask[n] == 0) continue;
+    const int32_t y = c.tokens[n];
+    if (y < 0 || y >= c.vocab) continue;
+    const float4 ws = reinterpret_cast<const float4 *>(row_ws)[n];
+    const double d = (double)ws.w;
+    cnt += 1.0;
+    sk3 += exp(d) * d - expm1(d);  // rho log rho - (rho - 1), Eq. 10 integrand
+    skl += (double)ws.z;
+  }
+  sh[0][threadIdx.x] = cnt;
+  sh[1][threadIdx.x] = sk3;
+  sh[2][threadIdx.x] = skl;
+  __syncthreads();
+  for (int off = kSegThreads / 2; off > 0; off >>= 1) {
+    if (threadIdx.x < off) {
+      sh[0][threadIdx.x] += sh[0][threadIdx.x + off];
+      sh[1][threadIdx.x] += sh[1][threadIdx.x + off];
+      sh[2][threadIdx.x] += sh[2][threadIdx.x + off];
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    if (mode == 0) {
+      double *a = out + 4 * (int64_t)i;
+      a[FOPD_ACC_CNT] += sh[0][0];
+      a[FOPD_ACC_K3] += sh[1][0];
+      a[FOPD_ACC_KL] += sh[2][0];
+      a[FOPD_ACC_ROWS] += (double)(hi - lo);
+    } else {
+      double *a = out + 2 * (int64_t)i;
+      a[0] += sh[2][0];
+      a[1] += sh[1][0];
+    }
+  }
+}
+
+// a6: freshness, gate, alignment ratio, per-token weight.  Single block.
+__global__ void __launch_bounds__(256)
+    freshness_kernel(const double *acc, const int32_t *tau, const int32_t *H, const float *d_sup,
+                     int32_t B, fopd_params p, float *f, float *w, float *d_roll, float *l_distill,
+                     float *m_align, float *coef, float *buffer_means, int32_t *status) {
+  __shared__ double sh[2][256];
+  double sum_f = 0.0, sum_m = 0.0;
+  for (int32_t i = threadIdx.x; i < B; i += 256) {
+    const double cnt = acc[4 * (int64_t)i + FOPD_ACC_CNT];
+    const int32_t t = tau[i], h = H[i];
+    if (t < 0 && status) atomicOr(status, FOPD_DEV_BAD_TAU);
+    if ((h <= 0 || cnt > (double)h) && status) atomicOr(status, FOPD_DEV_BAD_LENGTH);
+    double fi = 0.0, wi = 0.0, dr = 0.0, li = 0.0, mi = 0.0, ci = 0.0;
+    if (cnt > 0.0 && h > 0 && t >= 0) {
+      dr = acc[4 * (int64_t)i + FOPD_ACC_K3] / cnt;
+      li = acc[4 * (int64_t)i + FOPD_ACC_KL] / cnt;
+      const double ds = d_sup ? (double)d_sup[i] : 0.0;
+      const double surrogate = (double)p.alpha * sqrt(fmax(dr, 0.0)) + (double)p.beta * sqrt(fmax(ds, 0.0));
+      fi = exp(-surrogate) / ((double)t + 1.0);
+      wi = fmax(fi - (double)p.xi, 0.0);
+      mi = cnt / (double)h;
+      ci = wi / ((double)B * cnt);
+    }
+    if (f) f[i] = (float)fi;
+    if (w) w[i] = (float)wi;
+    if (d_roll) d_roll[i] = (float)dr;
+    if (l_distill) l_distill[i] = (float)li;
+    if (m_align) m_align[i] = (float)mi;
+    coef[i] = (float)ci;
+    sum_f += fi;
+    sum_m += mi;
+  }
+  if (buffer_means) {
+    sh[0][threadIdx.x] = sum_f;
+    sh[1][threadIdx.x] = sum_m;
+    __syncthreads();
+    for (int off = 128; off > 0; off >>= 1) {
+      if (threadIdx.x < off) {
+        sh[0][threadIdx.x] += sh[0][threadIdx.x + off];
+        sh[1][threadIdx.x] += sh[1][threadIdx.x + off];
+      }
+      __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+      buffer_means[0] = (float)(sh[0][0] / (double)B);
+      buffer_means[1] = (float)(sh[1][0] / (double)B);
+    }
+  }
+}
+
+// a7: L_i = w_i (l_i + lambda D_roll_i), L = (1/B) sum_i L_i.  Single block.
+__global__ void __launch_bounds__(256)
+    finalize_kernel(const double *loss_acc, const double *acc, const float *w, int32_t B, float lambda,
+                    float *per_sample, float *loss_out) {
+  __shared__ double sh[256];
+  double s = 0.0;
+  for (int32_t i = threadIdx.x; i < B; i += 256) {
+    const double cnt = acc[4 * (int64_t)i + FOPD_ACC_CNT];
+    double Li = 0.0;
+    if (cnt > 0.0 && w[i] > 0.f)
+      Li = (double)w[i] * (loss_acc[2 * (int64_t)i] + (double)lambda * loss_acc[2 * (int64_t)i + 1]) / cnt;
+    if (per_sample) per_sample[i] = (float)Li;
+    s += Li;
+  }
+  sh[threadIdx.x] = s;
+  __syncthreads();
+  for (int off = 128; off > 0; off >>= 1) {
+    if (threadIdx.x < off) sh[threadIdx.x] += sh[threadIdx.x + off];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) loss_out[0] = (float)(sh[0] / (double)B);
+}
+
+}  // namespace fopd

@@ -59,6 +59,11 @@ class Workload:
 DEFAULT_PARAMS = dict(alpha=1.0, beta=1.0, xi=0.15, lam=0.1)
 
 
+def _scaled_vocab(full: int, scale: float) -> int:
+    """Scaled vocabulary, kept a multiple of 8 so that bf16 rows stay 16-byte aligned."""
+    return max(96, (int(full * scale) + 7) // 8 * 8)
+
+
 def _packed(lengths):
     sid = np.repeat(np.arange(len(lengths), dtype=np.int32), lengths)
     return sid
@@ -68,7 +73,7 @@ def tiny(scale: float = 1.0) -> Workload:
     """Config 1: 4 x 256 tokens, V = 32,000, fp32, mask all ones, staleness 0..3."""
     rng = np.random.RandomState(0)
     B, T = 4, max(8, int(256 * scale))
-    V = max(64, int(32000 * scale))
+    V = _scaled_vocab(32000, scale)
     lengths = np.full(B, T, dtype=np.int64)
     sid = _packed(lengths)
     return Workload("tiny", B, V, torch.float32, sid.shape[0], sid, np.ones_like(sid, dtype=np.uint8),
@@ -81,7 +86,7 @@ def reasoning(scale: float = 1.0, V: int | None = None) -> Workload:
     padding masked, V = 151,936, bf16, staleness 0..2."""
     rng = np.random.RandomState(1)
     B, T = 16, max(16, int(2048 * scale))
-    V = V or max(96, int(151936 * scale))
+    V = V or _scaled_vocab(151936, scale)
     lengths = rng.randint(max(1, T // 4), T + 1, size=B)
     sid = np.repeat(np.arange(B, dtype=np.int32), T)
     pos = np.tile(np.arange(T), B)
@@ -96,7 +101,7 @@ def tool_use(scale: float = 1.0, V: int | None = None) -> Workload:
     staleness 0..4; streamed in 16,384-row chunks that cut across samples."""
     rng = np.random.RandomState(2)
     B = 32
-    V = V or max(96, int(151936 * scale))
+    V = V or _scaled_vocab(151936, scale)
     lo, hi = max(4, int(1024 * scale)), max(8, int(8192 * scale))
     lengths = rng.randint(lo, hi + 1, size=B)
     sid = _packed(lengths)
@@ -120,7 +125,7 @@ def coding_agent(scale: float = 1.0, V: int | None = None) -> Workload:
     16,384-row chunks."""
     rng = np.random.RandomState(3)
     B = 8
-    V = V or max(96, int(151936 * scale))
+    V = V or _scaled_vocab(151936, scale)
     lo, hi = max(8, int(16384 * scale)), max(16, int(32768 * scale))
     lengths = rng.randint(lo, hi + 1, size=B)
     sid = _packed(lengths)

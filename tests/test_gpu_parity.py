@@ -1,0 +1,199 @@
+"""GPU parity: the CUDA library against the fp64 CPU oracle, element by element,
+on the same seeded inputs, through the C ABI (via the ctypes binding)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2605_17862_b200 import binding as fb
+from paper_2605_17862_b200 import pipeline as pl
+from paper_2605_17862_b200 import synth
+
+import _parity as par
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _chunks(wl, row_stride=None):
+    return [synth.gen_chunk(wl, j, DEV, row_stride=row_stride) for j in range(wl.n_chunks)]
+
+
+@pytest.mark.parametrize("use_row_ws", [True, False])
+def test_tiny_config_full_size(use_row_ws):
+    wl = synth.tiny()  # 4 x 256 rows, V = 32,000, fp32, single chunk, seed 0
+    out = par.compare(_chunks(wl), wl.B, wl.tau, wl.H, use_row_ws=use_row_ws)
+    print("tiny", out)
+
+
+@pytest.mark.parametrize("name,scale", [("reasoning", 1 / 16), ("tool_use", 1 / 16), ("coding_agent", 1 / 16)])
+@pytest.mark.parametrize("use_row_ws", [True, False])
+def test_scaled_workloads(name, scale, use_row_ws):
+    wl = synth.WORKLOADS[name](scale=scale)  # V = 9,496: many vectors per thread, several chunks
+    out = par.compare(_chunks(wl), wl.B, wl.tau, wl.H, use_row_ws=use_row_ws, grad_rows_per_chunk=64)
+    print(name, wl.n_rows, wl.V, out)
+
+
+@pytest.mark.parametrize("V,stride", [(1, 8), (2, 8), (5, 8), (7, 8), (33, 40), (1000, 1000), (9501, 9504),
+                                      (4099, 4104)])
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_odd_vocabularies_and_pitch(V, stride, dtype):
+    """Ragged tails: vocabularies that do not fill the last 16-byte vector, a row
+    pitch larger than the vocabulary, and single-digit vocabularies."""
+    rng = np.random.RandomState(V)
+    B, n = 3, 37
+    lengths = np.array([10, 15, 12])
+    sid = np.repeat(np.arange(B, dtype=np.int32), lengths)
+    mask = (rng.rand(n) > 0.2).astype(np.uint8)
+    wl = synth.Workload("odd", B, V, dtype, n, sid, mask, np.array([0, 1, 2], np.int32),
+                        lengths.astype(np.int32), sigma_s=2.0, seed=V)
+    ch = synth.gen_chunk(wl, 0, DEV, row_stride=stride)
+    # poison the pitch padding: it must be neither read into results nor written
+    ch["student"][:, V:] = 1e4
+    ch["teacher"][:, V:] = -1e4
+    for use_ws in (True, False):
+        par.compare([ch], B, wl.tau, wl.H, use_row_ws=use_ws, vocab=V)
+
+
+def test_single_row_and_empty_chunk():
+    wl = synth.Workload("one", 1, 64, torch.bfloat16, 1, np.zeros(1, np.int32), np.ones(1, np.uint8),
+                        np.zeros(1, np.int32), np.ones(1, np.int32), seed=5)
+    ch = synth.gen_chunk(wl, 0, DEV)
+    par.compare([ch], 1, wl.tau, wl.H)
+    # an empty chunk between two real ones changes nothing
+    empty = {k: v[:0] for k, v in ch.items()}
+    a = par.gpu_run([ch], 1, wl.tau, wl.H)
+    b = par.gpu_run([empty, ch], 1, wl.tau, wl.H)
+    assert torch.equal(a[0].acc, b[0].acc) and torch.equal(a[0].loss, b[0].loss)
+    assert torch.equal(a[2][0], b[2][1])
+
+
+def test_fully_masked_sample_and_gated_sample():
+    wl = synth.reasoning(scale=1 / 32)
+    wl.mask[wl.sample_id == 3] = 0           # no aligned token: invalid, f = w = m = 0 (Algorithm 1)
+    wl.tau = wl.tau.copy()
+    wl.tau[5] = 40                           # far below the gate: w = 0, gradient rows exactly zero
+    out = par.compare(_chunks(wl), wl.B, wl.tau, wl.H)
+    buf, _, dl, _ = par.gpu_run(_chunks(wl), wl.B, wl.tau, wl.H)
+    assert float(buf.f[3]) == 0 and float(buf.w[3]) == 0 and float(buf.m_align[3]) == 0
+    assert float(buf.f[5]) > 0 and float(buf.w[5]) == 0 and float(buf.per_sample_loss[5]) == 0
+    rows5 = torch.as_tensor(wl.sample_id == 5, device=DEV)
+    assert float(dl[0][rows5].abs().max()) == 0.0
+
+
+def test_bad_ids_set_status_bits_and_are_treated_as_masked():
+    wl = synth.tiny(scale=1 / 8)
+    ch = synth.gen_chunk(wl, 0, DEV)
+    ch["tokens"][3] = -1
+    ch["tokens"][4] = wl.V
+    par.compare([ch], wl.B, wl.tau, wl.H, expect_bits=fb_bits("token"))
+    ch = synth.gen_chunk(wl, 0, DEV)
+    ch["sample_id"][-1] = wl.B  # keeps the array non-decreasing
+    par.compare([ch], wl.B, wl.tau, wl.H, expect_bits=fb_bits("sample"))
+    tau = wl.tau.copy()
+    tau[1] = -2
+    H = wl.H.copy()
+    H[2] = 0
+    par.compare([synth.gen_chunk(wl, 0, DEV)], wl.B, tau, H, expect_bits=fb_bits("tau") | fb_bits("length"))
+
+
+def fb_bits(kind):
+    return {"token": 1, "sample": 2, "tau": 4, "length": 8}[kind]
+
+
+def test_teacher_equals_student_gives_zero_kl_exactly():
+    wl = synth.reasoning(scale=1 / 32)
+    ch = synth.gen_chunk(wl, 0, DEV)
+    ch["teacher"] = ch["student"].clone()
+    buf, rows, dl, bits = par.gpu_run([ch], wl.B, wl.tau, wl.H)
+    assert float(rows[0].kl.abs().max()) == 0.0
+    assert torch.equal(rows[0].lp_s, rows[0].lp_t)
+    par.compare([ch], wl.B, wl.tau, wl.H)
+    # with the anchor off as well the gradient vanishes identically
+    p0 = dict(par.PARAMS, lam=0.0)
+    _, _, dl0, _ = par.gpu_run([ch], wl.B, wl.tau, wl.H, params=p0)
+    assert float(dl0[0].abs().max()) == 0.0
+
+
+def test_d_sup_input_and_lag_only_freshness():
+    wl = synth.tool_use(scale=1 / 32)
+    chunks = _chunks(wl)
+    d_sup = np.linspace(0.0, 0.3, wl.B).astype(np.float32)
+    par.compare(chunks, wl.B, wl.tau, wl.H, d_sup=d_sup, params=dict(alpha=0.7, beta=2.0, xi=0.1, lam=0.3),
+                grad_rows_per_chunk=16)
+    # alpha = beta = 0: the lag-only baseline f = 1 / (tau + 1) (Appendix B)
+    buf, *_ = par.gpu_run(chunks, wl.B, wl.tau, wl.H, params=dict(alpha=0.0, beta=0.0, xi=0.0, lam=0.0))
+    assert np.allclose(buf.f.cpu().numpy(), 1.0 / (wl.tau + 1.0), rtol=1e-7)
+
+
+def test_cached_and_uncached_paths_agree_and_reruns_are_bit_identical():
+    wl = synth.coding_agent(scale=1 / 32)
+    chunks = _chunks(wl)
+    a = par.gpu_run(chunks, wl.B, wl.tau, wl.H, use_row_ws=True)
+    b = par.gpu_run(chunks, wl.B, wl.tau, wl.H, use_row_ws=True)
+    c = par.gpu_run(chunks, wl.B, wl.tau, wl.H, use_row_ws=False)
+    assert torch.equal(a[0].acc, b[0].acc) and torch.equal(a[0].loss_acc, b[0].loss_acc)
+    assert torch.equal(a[0].loss, b[0].loss) and torch.equal(a[0].f, b[0].f)
+    for x, y in zip(a[2], b[2]):
+        assert torch.equal(x, y)
+    assert torch.allclose(a[0].loss, c[0].loss, rtol=1e-5)
+    for x, y in zip(a[2], c[2]):
+        assert torch.allclose(x.float(), y.float(), rtol=2e-2, atol=1e-7)
+
+
+def test_chunk_split_invariance_on_gpu():
+    wl = synth.tool_use(scale=1 / 32)
+    whole = synth.gen_chunk(wl, 0, DEV) if wl.n_chunks == 1 else None
+    chunks = _chunks(wl)
+    cat = {k: torch.cat([c[k] for c in chunks]) for k in chunks[0]}
+    a = par.gpu_run([cat], wl.B, wl.tau, wl.H)
+    for cut in (1, 777, cat["student"].shape[0] - 1):
+        parts = [{k: v[:cut] for k, v in cat.items()}, {k: v[cut:] for k, v in cat.items()}]
+        b = par.gpu_run(parts, wl.B, wl.tau, wl.H)
+        assert torch.equal(a[0].acc[:, 0], b[0].acc[:, 0])
+        assert torch.allclose(a[0].acc, b[0].acc, rtol=1e-12)
+        assert torch.allclose(a[0].f, b[0].f, rtol=1e-6) and torch.allclose(a[0].loss, b[0].loss, rtol=1e-6)
+        assert torch.equal(torch.cat(b[2]), a[2][0]) or torch.allclose(torch.cat(b[2]).float(), a[2][0].float(),
+                                                                       rtol=2e-2, atol=1e-9)
+
+
+def test_outputs_do_not_overrun():
+    """Canary rows around dlogits and the per-row outputs stay untouched."""
+    wl = synth.reasoning(scale=1 / 32)
+    ch = synth.gen_chunk(wl, 0, DEV)
+    n, V = ch["student"].shape
+    big = torch.full((n + 2, V), 7.0, dtype=ch["student"].dtype, device=DEV)
+    buf = pl.BatchBuffers(wl.B, DEV)
+    rows = pl.RowOutputs.alloc(n + 2, DEV)
+    for t in (rows.lp_s, rows.lp_t, rows.kl, rows.ratio, rows.row_ws):
+        t.fill_(7.0)
+    view = pl.RowOutputs(rows.lp_s[1:-1], rows.lp_t[1:-1], rows.kl[1:-1], rows.ratio[1:-1], rows.row_ws[1:-1])
+    p = fb.params(**par.PARAMS)
+    tau = torch.as_tensor(wl.tau, device=DEV)
+    H = torch.as_tensor(wl.H, device=DEV)
+    pl.step([pl.to_chunk(ch)], [big[1:-1]], buf, tau, H, None, p, [view])
+    torch.cuda.synchronize()
+    assert float((big[0] - 7).abs().max()) == 0 and float((big[-1] - 7).abs().max()) == 0
+    for t in (rows.lp_s, rows.lp_t, rows.kl, rows.ratio):
+        assert float(t[0]) == 7.0 and float(t[-1]) == 7.0
+    assert float((rows.row_ws[0] - 7).abs().max()) == 0 and float((rows.row_ws[-1] - 7).abs().max()) == 0
+
+
+def test_host_validation_errors():
+    wl = synth.tiny(scale=1 / 8)
+    ch = synth.gen_chunk(wl, 0, DEV)
+    buf = pl.BatchBuffers(wl.B, DEV)
+    p = fb.params(**par.PARAMS)
+    dl = torch.empty_like(ch["student"])
+    with pytest.raises(fb.FopdError) as e:  # dlogits aliases student
+        fb.fopd_loss_fwd_bwd(pl.to_chunk(ch), wl.B, buf.coef, p, ch["student"], buf.loss_acc)
+    assert e.value.code == -7
+    with pytest.raises(fb.FopdError) as e:  # negative alpha
+        fb.fopd_loss_fwd_bwd(pl.to_chunk(ch), wl.B, buf.coef, fb.params(alpha=-1.0), dl, buf.loss_acc)
+    assert e.value.code == -5
+    mis = dict(ch, student=ch["student"].view(-1)[1:1 + (ch["student"].shape[0] - 1) * wl.V].view(-1, wl.V),
+               teacher=ch["teacher"][:-1])
+    mis = {k: (v if k in ("student", "teacher") else v[:-1]) for k, v in mis.items()}
+    c = pl.to_chunk(dict(mis, teacher=mis["student"]))
+    with pytest.raises(fb.FopdError) as e:  # base not 16-byte aligned
+        fb.fopd_token_stats(c, wl.B, buf.acc)
+    assert e.value.code == -2
