@@ -1,0 +1,362 @@
+#!/usr/bin/env python
+"""Benchmark of the f-OPD loss hot path (libfopd) on B200.
+
+One step = one pass of the whole path over one batch of synthetic input:
+fopd_token_stats on every chunk, fopd_sample_freshness, fopd_loss_fwd_bwd on
+every chunk, fopd_loss_finalize.  Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl fopd|reference]
+                  [--workload reasoning|tiny|tool_use|coding_agent|roofline:<rows>x<V>]
+                  [--path cached|standalone]
+
+N > 1 (under torchrun): the path has no exchange step, so every rank runs an
+independent replica of the workload (different seed); time is the max over
+ranks, value the sum of tokens over ranks divided by it ("weak" scaling).
+--impl reference times the fp64 CPU oracle on a bounded sample of the same
+workload on the host cores (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "fused OPD loss path (token stats + freshness + loss fwd+bwd) throughput at V=151,936"
+UNIT = "tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant
+# kernel from an ncu capture, keyed by (kernel, workload); see profiles/.  None = not captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="fopd", choices=["fopd", "reference"])
+    ap.add_argument("--workload", default="reasoning")
+    ap.add_argument("--path", default="cached", choices=["cached", "standalone"])
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-sample-rows", type=int, default=0, help="rows of the CPU-oracle sample (0 = auto)")
+    return ap.parse_args()
+
+
+def make_workload(name: str):
+    from paper_2605_17862_b200 import synth
+
+    if name.startswith("roofline:"):
+        rows, V = name.split(":")[1].split("x")
+        return synth.roofline_point(int(rows), int(V))
+    return synth.WORKLOADS[name]()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+                pw.append(float(r[2]))
+            except Exception:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def algorithmic_bytes(wl, active_rows: int):
+    """Minimum bytes: statistics sweep reads S and T of aligned rows; the loss
+    fwd+bwd reads S and T of differentiated rows once and writes every dlogits row."""
+    e = 2 if str(wl.dtype).endswith("bfloat16") else 4
+    aligned = int(wl.mask.sum())
+    row = wl.V * e
+    stats = 2 * row * aligned
+    grad = 3 * row * active_rows + row * (wl.n_rows - active_rows)
+    return stats, grad
+
+
+def run_reference(args, rank: int):
+    """CPU oracle on a bounded sample of the workload (rank 0 only)."""
+    if rank != 0:
+        return
+    import numpy as np
+    import torch
+    from oracle import fopd_oracle as orc
+    from paper_2605_17862_b200 import synth
+
+    wl = make_workload(args.workload)
+    res = time_oracle(wl, args.cpu_sample_rows or 256, steps=args.steps, warmup=args.warmup)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": res["ms_per_step"], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "rows": wl.n_rows, "vocab": wl.V, "samples": wl.B, "sample": res["sample"]},
+        "cpu_baseline": {"value": res["value"], "unit": UNIT, "cores": res["cores"], "kind": "oracle",
+                         "sample": res["sample"]},
+        "e2e": {"value": res["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def time_oracle(wl, sample_rows: int, steps: int = 1, warmup: int = 0):
+    """Times the oracle, as it stands, on the first `sample_rows` aligned rows of
+    chunk 0: the statistics pass, per-sample sums, freshness, loss and the
+    gradient of every sampled row (the same steps the GPU path runs)."""
+    import numpy as np
+    from oracle import fopd_oracle as orc
+    from paper_2605_17862_b200 import synth
+
+    lo, hi = wl.chunk_range(0)
+    aligned = np.nonzero(wl.mask[lo:hi])[0][:sample_rows]
+    n = int(aligned.max()) + 1 if len(aligned) else 0
+    sub = synth.Workload(wl.name, wl.B, wl.V, wl.dtype, n, wl.sample_id[:n], wl.mask[:n], wl.tau, wl.H,
+                         wl.sigma_s, wl.boost_frac, wl.boost, wl.sigma_t, wl.sigma_b, wl.seed)
+    ch = synth.gen_chunk(sub, 0, "cpu", row_block=64)
+    P = synth.DEFAULT_PARAMS
+    times = []
+    for it in range(warmup + steps):
+        t0 = time.perf_counter()
+        r = orc.run_batch([ch], wl.B, wl.tau, wl.H, None, P["alpha"], P["beta"], P["xi"], P["lam"])
+        orc.grad_rows(ch["student"], ch["teacher"], ch["tokens"], ch["behav_logprob"], ch["mask"],
+                      ch["sample_id"], r.fresh.coef, P["lam"], aligned)
+        if it >= warmup:
+            times.append(time.perf_counter() - t0)
+    dt = sum(times) / len(times)
+    return {"value": len(aligned) / dt, "ms_per_step": dt * 1e3, "cores": orc.num_threads(),
+            "sample": f"first {len(aligned)} aligned rows of chunk 0 ({n} rows incl. masked), V={wl.V}, "
+                      f"stats + freshness + loss + gradient of every sampled row"}
+
+
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    from paper_2605_17862_b200 import binding as fb
+    from paper_2605_17862_b200 import pipeline as pl
+    from paper_2605_17862_b200 import synth
+
+    fb.lib()  # fail loudly if the CUDA library is missing
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    wl = make_workload(args.workload)
+    wl.seed = wl.seed + 100 * rank  # independent replica per rank
+    chunks_d = [synth.gen_chunk(wl, j, dev) for j in range(wl.n_chunks)]
+    chunks = [pl.to_chunk(c) for c in chunks_d]
+    dlogits = [torch.empty_like(c["student"]) for c in chunks_d]
+    rows = [pl.RowOutputs.alloc(c["student"].shape[0], dev) for c in chunks_d]
+    buf = pl.BatchBuffers(wl.B, dev)
+    P = synth.DEFAULT_PARAMS
+    p = fb.params(**P)
+    tau = torch.as_tensor(wl.tau, device=dev)
+    H = torch.as_tensor(wl.H, device=dev)
+    cached = args.path == "cached"
+
+    def one_step(ev=None):
+        buf.reset()
+        if ev: ev[0].record()
+        pl.measure(chunks, buf, rows, keep_row_ws=cached)
+        if ev: ev[1].record()
+        pl.freshness(buf, tau, H, None, p)
+        if ev: ev[2].record()
+        pl.optimise(chunks, dlogits, buf, p, rows, use_row_ws=cached)
+        if ev: ev[3].record()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        one_step()
+    barrier()
+    assert fb.fopd_check_status(buf.status) == 0
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    t_begin.record()
+    for k in range(args.steps):
+        one_step(events[k])
+    t_end.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = t_begin.elapsed_time(t_end)
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t[0])
+    stats_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in events) / len(chunks)
+    grad_ms = statistics.mean(e[2].elapsed_time(e[3]) for e in events) / len(chunks)
+
+    coef = buf.coef.cpu().numpy()
+    active_rows = int(((coef[np.clip(wl.sample_id, 0, wl.B - 1)] > 0) & (wl.mask > 0)).sum())
+    aligned = int(wl.mask.sum())
+    stats_bytes, grad_bytes = algorithmic_bytes(wl, active_rows)
+    ms_per_step = total_ms / args.steps
+    value = world * aligned / (ms_per_step * 1e-3)
+    peak, peak_src = measured_peak()
+    n_launch_chunk = len(chunks)
+    kernels_per_step = n_launch_chunk * (2 + (2 if cached else 3)) + 2
+    grad_kernel = "grad_stream_kernel" if cached else "token_stats_kernel+grad_stream_kernel"
+    achieved = grad_bytes / n_launch_chunk / (grad_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {
+            "workload": wl.name, "rows": wl.n_rows, "aligned_tokens": aligned, "differentiated_rows": active_rows,
+            "vocab": wl.V, "samples": wl.B, "logits_dtype": str(wl.dtype).replace("torch.", ""),
+            "chunks": len(chunks), "path": args.path, "tokens_counted": "aligned (mask = 1) rows",
+            "l2": "inputs (2 x %.2f GB) far larger than the 126 MB L2, no flush needed" %
+                  (wl.n_rows * wl.V * (2 if wl.dtype == torch.bfloat16 else 4) / 1e9),
+            "parallelism": "replicas only" if world > 1 else "1 gpu", "params": P,
+        },
+        "gpu_launches": kernels_per_step * args.steps,
+        "phases_ms": {"token_stats_per_chunk": stats_ms, "loss_fwd_bwd_per_chunk": grad_ms,
+                      "freshness": statistics.mean(e[1].elapsed_time(e[2]) for e in events)},
+        "token_stats": {"gbs": stats_bytes / n_launch_chunk / (stats_ms * 1e-3) / 1e9,
+                        "frac_of_peak": stats_bytes / n_launch_chunk / (stats_ms * 1e-3) / 1e9 / peak},
+        "loss_fwd_bwd": {"tokens_per_s": active_rows / n_launch_chunk / (grad_ms * 1e-3), "gbs": achieved,
+                         "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS},
+        "roofline": {"bound": "hbm", "kernel": grad_kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_source": peak_src,
+                     "traffic": NCU_TRAFFIC_BYTES.get((grad_kernel, wl.name)),
+                     "algorithmic_bytes_per_launch": grad_bytes / n_launch_chunk},
+        "clocks": clocks,
+        "loss": float(buf.loss.cpu()[0]),
+    }
+
+    # ---- end to end through the host-buffer entry point (pinned host memory, copies timed)
+    if not args.no_e2e and len(chunks) >= 1:
+        try:
+            line["e2e"] = run_e2e(args, wl, chunks_d, dev, world, aligned)
+        except Exception as exc:  # report, never fake
+            line["e2e"] = {"value": None, "unit": UNIT, "error": repr(exc)[:200]}
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        res = time_oracle(wl, args.cpu_sample_rows or 512)
+        line["cpu_baseline"] = {"value": res["value"], "unit": UNIT, "cores": res["cores"], "kind": "oracle",
+                                "sample": res["sample"]}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(args, wl, chunks_d, dev, world, aligned):
+    """Same step through fopd_step_host: logits start in pinned host memory, every step
+    uploads them, runs the path and downloads dlogits and the per-sample results."""
+    import torch
+    import torch.distributed as dist
+    from paper_2605_17862_b200 import binding as fb
+    from paper_2605_17862_b200 import pipeline as pl
+    from paper_2605_17862_b200 import synth
+
+    host = []
+    for c in chunks_d:
+        host.append({k: v.cpu().pin_memory() for k, v in c.items()})
+    hchunks = [pl.to_chunk(c) for c in host]
+    hdl = [torch.empty_like(c["student"]).pin_memory() for c in host]
+    need = fb.fopd_step_host_workspace_bytes(hchunks, wl.B, True)
+    free, _ = torch.cuda.mem_get_info(dev)
+    if need > free - (2 << 30):
+        need = fb.fopd_step_host_workspace_bytes(hchunks, wl.B, False)
+    ws = torch.empty(need, dtype=torch.uint8, device=dev)
+    tau = torch.as_tensor(wl.tau)
+    H = torch.as_tensor(wl.H)
+    p = fb.params(**synth.DEFAULT_PARAMS)
+    fb.fopd_step_host(hchunks, wl.B, tau, H, None, p, hdl, ws)  # warm-up
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.e2e_steps):
+        res = fb.fopd_step_host(hchunks, wl.B, tau, H, None, p, hdl, ws)
+    torch.cuda.synchronize()
+    dt = (time.perf_counter() - t0) / args.e2e_steps
+    if world > 1:
+        t = torch.tensor([dt], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dt = float(t[0])
+    logit_bytes = sum(c["student"].numel() * c["student"].element_size() for c in host)
+    side = sum(c["tokens"].numel() * 13 for c in host)
+    resident = need == fb.fopd_step_host_workspace_bytes(hchunks, wl.B, True)
+    return {"value": world * aligned / dt, "unit": UNIT, "ms_per_step": dt * 1e3,
+            "h2d_bytes_per_step": (2 if resident else 4) * logit_bytes + side,
+            "d2h_bytes_per_step": logit_bytes + 7 * 4 * wl.B + 16,
+            "steps": args.e2e_steps, "api": "fopd_step_host (pinned host buffers)", "loss": float(res["loss"][0])}
+
+
+if __name__ == "__main__":
+    main()

@@ -199,6 +199,45 @@ int fopd_loss_finalize(const double *loss_acc, const double *acc, const float *w
  * FOPD_ERR_CUDA. */
 int fopd_check_status(const int32_t *status, int32_t *bits_out /* HOST */, void *stream);
 
+/*
+ * Whole batch from HOST memory: the calling sequence above (statistics for every
+ * chunk, freshness, fused loss forward + backward for every chunk, finalize;
+ * Algorithm 1's measurement and optimisation phases) with the host<->device
+ * copies done by the library.  For callers whose logits live in host memory
+ * (pinned memory copies fastest).
+ *
+ *   chunks      HOST array of n_chunks descriptors whose pointers are HOST
+ *               pointers (same layout rules as for device chunks)
+ *   staleness, seq_len, d_sup   HOST [B] (d_sup may be NULL)
+ *   dlogits     HOST array of n_chunks HOST pointers; dlogits[j] receives
+ *               chunk j's gradient, [n_rows_j, vocab] at the chunk's pitch
+ *   out         HOST outputs, [B] each (any may be NULL) and loss[1] (required);
+ *               status_bits[1] receives the device status word
+ *   workspace   DEVICE scratch owned by the caller, 256-byte aligned, at least
+ *               fopd_step_host_workspace_bytes(.., resident = 0) bytes.  If it
+ *               is at least the resident = 1 size, all logits stay on the device
+ *               between the two phases and are uploaded once; otherwise every
+ *               chunk is uploaded twice (once per phase).
+ *
+ * Synchronises `stream` before returning.  Returns FOPD_ERR_SIZE if the
+ * workspace is too small, FOPD_ERR_DEVICE if the status word is non-zero (the
+ * outputs are still written).
+ */
+typedef struct {
+  float *f, *w, *d_roll, *l_distill, *m_align, *per_sample_loss; /* [B] or NULL */
+  float *buffer_means;                                            /* [2] or NULL */
+  float *loss;                                                    /* [1]         */
+  int32_t *status_bits;                                           /* [1] or NULL */
+} fopd_host_outputs;
+
+uint64_t fopd_step_host_workspace_bytes(const fopd_chunk *chunks /* HOST */, int32_t n_chunks,
+                                        int32_t B, int32_t resident);
+
+int fopd_step_host(const fopd_chunk *chunks /* HOST */, int32_t n_chunks, int32_t B,
+                   const int32_t *staleness, const int32_t *seq_len, const float *d_sup,
+                   fopd_params p, void *const *dlogits, const fopd_host_outputs *out,
+                   void *workspace, uint64_t workspace_bytes, void *stream);
+
 const char *fopd_strerror(int code);
 int fopd_version(void);
 

@@ -18,7 +18,7 @@ FOPD_BF16, FOPD_F32 = 0, 1
 
 EXPORTS = (
     "fopd_token_stats", "fopd_sample_freshness", "fopd_loss_fwd_bwd", "fopd_loss_finalize",
-    "fopd_check_status", "fopd_strerror", "fopd_version",
+    "fopd_check_status", "fopd_strerror", "fopd_version", "fopd_step_host", "fopd_step_host_workspace_bytes",
 )
 
 
@@ -42,6 +42,12 @@ class fopd_chunk(ctypes.Structure):
     ]
 
 
+class fopd_host_outputs(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in
+                ("f", "w", "d_roll", "l_distill", "m_align", "per_sample_loss", "buffer_means", "loss",
+                 "status_bits")]
+
+
 _lib = None
 
 
@@ -63,6 +69,11 @@ def lib() -> ctypes.CDLL:
         L.fopd_loss_fwd_bwd.argtypes = [ctypes.POINTER(fopd_chunk), i32, vp, vp, fopd_params, vp, vp, vp, vp]
         L.fopd_loss_finalize.argtypes = [vp, vp, vp, i32, fopd_params, vp, vp, vp]
         L.fopd_check_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
+        L.fopd_step_host_workspace_bytes.restype = ctypes.c_uint64
+        L.fopd_step_host_workspace_bytes.argtypes = [ctypes.POINTER(fopd_chunk), i32, i32, i32]
+        L.fopd_step_host.argtypes = [ctypes.POINTER(fopd_chunk), i32, i32, vp, vp, vp, fopd_params,
+                                     ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(fopd_host_outputs), vp,
+                                     ctypes.c_uint64, vp]
         for name in EXPORTS:
             getattr(L, name)
         _lib = L
@@ -163,3 +174,34 @@ def fopd_check_status(status, stream=None) -> int:
     if rc not in (0, -8):
         raise FopdError(rc, "fopd_check_status")
     return int(bits.value)
+
+
+def _chunk_array(chunks):
+    arr = (fopd_chunk * len(chunks))()
+    for j, ch in enumerate(chunks):
+        arr[j] = ch.c_struct()
+    return arr
+
+
+def fopd_step_host_workspace_bytes(chunks, B: int, resident: bool) -> int:
+    """Device workspace size fopd_step_host needs for these HOST chunks."""
+    return int(lib().fopd_step_host_workspace_bytes(_chunk_array(chunks), len(chunks), B, int(resident)))
+
+
+def fopd_step_host(chunks, B: int, staleness, seq_len, d_sup, p: fopd_params, dlogits, workspace, *,
+                   stream=None) -> dict:
+    """Whole batch from HOST tensors (``chunks`` hold CPU tensors, ideally pinned;
+    ``dlogits`` is a list of CPU tensors receiving the gradients).  Returns the
+    per-sample outputs as CPU tensors plus the scalar loss and status bits."""
+    arr = _chunk_array(chunks)
+    z = lambda n: torch.zeros(n, dtype=torch.float32)
+    res = dict(f=z(B), w=z(B), d_roll=z(B), l_distill=z(B), m_align=z(B), per_sample_loss=z(B),
+               buffer_means=z(2), loss=z(1), status_bits=torch.zeros(1, dtype=torch.int32))
+    outs = fopd_host_outputs(*[res[n].data_ptr() for n, _ in fopd_host_outputs._fields_])
+    dl = (ctypes.c_void_p * len(dlogits))(*[d.data_ptr() for d in dlogits])
+    rc = lib().fopd_step_host(arr, len(chunks), B, _ptr(staleness), _ptr(seq_len), _ptr(d_sup), p, dl,
+                              ctypes.byref(outs), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                              _stream(stream))
+    if rc not in (0, -8):
+        raise FopdError(rc, "fopd_step_host")
+    return res
