@@ -1,0 +1,82 @@
+// Host-side helpers shared by the entry points of libfopd: argument checks,
+// device query and the launch of the statistics sweep.
+#pragma once
+
+#include <cmath>
+
+#include "stream_kernels.cuh"
+
+namespace fopd {
+
+struct DeviceInfo {
+  int sm_count = 0;
+};
+
+static inline int device_info(DeviceInfo *out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FOPD_ERR_CUDA;
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return FOPD_ERR_CUDA;
+  out->sm_count = sms;
+  return FOPD_OK;
+}
+
+static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static inline int check_chunk(const fopd_chunk *c, int32_t B) {
+  if (!c) return FOPD_ERR_NULL;
+  if (c->dtype != FOPD_BF16 && c->dtype != FOPD_F32) return FOPD_ERR_DTYPE;
+  if (c->n_rows < 0 || c->vocab <= 0 || c->row_stride < c->vocab || B <= 0) return FOPD_ERR_SIZE;
+  if (c->vocab > (int64_t)1 << 30 || c->n_rows > (int64_t)1 << 40) return FOPD_ERR_SIZE;
+  if (c->n_rows == 0) return FOPD_OK;
+  if (!c->student || !c->teacher || !c->behav_logprob || !c->tokens || !c->mask || !c->sample_id)
+    return FOPD_ERR_NULL;
+  const int64_t esz = c->dtype == FOPD_BF16 ? 2 : 4;
+  if (!aligned16(c->student) || !aligned16(c->teacher) || (c->row_stride * esz) % 16 != 0)
+    return FOPD_ERR_ALIGN;
+  return FOPD_OK;
+}
+
+static inline ChunkDev to_dev(const fopd_chunk *c) {
+  ChunkDev d;
+  d.student = c->student;
+  d.teacher = c->teacher;
+  d.behav = c->behav_logprob;
+  d.tokens = c->tokens;
+  d.mask = c->mask;
+  d.sid = c->sample_id;
+  d.n_rows = c->n_rows;
+  d.vocab = c->vocab;
+  d.stride = c->row_stride;
+  return d;
+}
+
+static inline int check_params(const fopd_params &p) {
+  if (!std::isfinite(p.alpha) || !std::isfinite(p.beta) || !std::isfinite(p.xi) || !std::isfinite(p.lambda))
+    return FOPD_ERR_PARAM;
+  if (p.alpha < 0.f || p.beta < 0.f) return FOPD_ERR_PARAM;
+  return FOPD_OK;
+}
+
+static inline int launch_ok() { return cudaGetLastError() == cudaSuccess ? FOPD_OK : FOPD_ERR_CUDA; }
+
+static inline int stream_grid(const DeviceInfo &di, int64_t n_rows) {
+  const int64_t persistent = (int64_t)di.sm_count * 2;  // two 512-thread CTAs per SM
+  return (int)(n_rows < persistent ? n_rows : persistent);
+}
+
+// Enqueues the statistics sweep of a chunk into row_ws (and the optional
+// per-row outputs).
+static inline int launch_stats(const fopd_chunk *c, int32_t B, float *lp_s, float *lp_t, float *kl, float *ratio,
+                 float *row_ws, int32_t *status, cudaStream_t st, const DeviceInfo &di) {
+  const ChunkDev d = to_dev(c);
+  const int grid = stream_grid(di, c->n_rows);
+  if (c->dtype == FOPD_BF16)
+    token_stats_kernel<FOPD_BF16><<<grid, kStreamThreads, 0, st>>>(d, B, lp_s, lp_t, kl, ratio, row_ws, status);
+  else
+    token_stats_kernel<FOPD_F32><<<grid, kStreamThreads, 0, st>>>(d, B, lp_s, lp_t, kl, ratio, row_ws, status);
+  return launch_ok();
+}
+
+
+}  // namespace fopd

@@ -240,7 +240,7 @@ __device__ __forceinline__ int64_t lower_bound_sid(const int32_t *sid, int64_t n
   return lo;
 }
 
-__global__ void __launch_bounds__(kSegThreads)
+static __global__ void __launch_bounds__(kSegThreads)
     segment_reduce_kernel(ChunkDev c, int32_t B, const float *row_ws, const float *coef, int mode,
                           double *out) {
   __shared__ double sh[3][kSegThreads];
@@ -288,7 +288,7 @@ __global__ void __launch_bounds__(kSegThreads)
 }
 
 // a6: freshness, gate, alignment ratio, per-token weight.  Single block.
-__global__ void __launch_bounds__(256)
+static __global__ void __launch_bounds__(256)
     freshness_kernel(const double *acc, const int32_t *tau, const int32_t *H, const float *d_sup,
                      int32_t B, fopd_params p, float *f, float *w, float *d_roll, float *l_distill,
                      float *m_align, float *coef, float *buffer_means, int32_t *status) {
@@ -338,7 +338,7 @@ __global__ void __launch_bounds__(256)
 }
 
 // a7: L_i = w_i (l_i + lambda D_roll_i), L = (1/B) sum_i L_i.  Single block.
-__global__ void __launch_bounds__(256)
+static __global__ void __launch_bounds__(256)
     finalize_kernel(const double *loss_acc, const double *acc, const float *w, int32_t B, float lambda,
                     float *per_sample, float *loss_out) {
   __shared__ double sh[256];
