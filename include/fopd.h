@@ -138,6 +138,39 @@ int fopd_token_stats(const fopd_chunk *chunk /* HOST */, int32_t B, float *lp_s,
                      double *acc, int32_t *status, void *stream);
 
 /*
+ * fopd_token_stats for callers that must not allocate device memory.  (The
+ * paper has no counterpart; this is an interface convenience.)
+ *
+ * Who needs it: a trainer that has handed all of the GPU's memory to its own
+ * allocator, so that the CUDA memory pool fopd_token_stats(row_ws = NULL) draws
+ * from may have nothing left; and code with a strict no-allocation rule inside
+ * its steady-state loop, where an allocation could stall on the device or fail
+ * in the middle of a step.  Such callers would otherwise have to carve a
+ * row_ws buffer out of their own memory.
+ *
+ * Same arguments, outputs and results as fopd_token_stats without the row_ws
+ * parameter: the per-row scratch lives in a fixed array compiled into the
+ * library, FOPD_STATIC_MAX_ROWS * 16 bytes = 1 MiB on every GPU that loads the
+ * library, held until the process exits.  The call makes no cudaMalloc,
+ * cudaFree or other allocating call.
+ *
+ *   - chunk->n_rows > FOPD_STATIC_MAX_ROWS returns FOPD_ERR_SIZE and enqueues
+ *     nothing; split the chunk.
+ *   - The first call on each device looks the array's device address up
+ *     (cudaGetSymbolAddress, with that device current) and caches it; make
+ *     that first call outside any stream capture.
+ *   - All calls on a device share the one array, which still holds the previous
+ *     call's values.  Nothing has to be cleared: each call overwrites the
+ *     entries of all its rows before it reads them.  Two calls whose kernels can
+ *     overlap on the GPU (different streams, or the same entry point from two
+ *     threads) race on the array; order them on one stream.
+ */
+#define FOPD_STATIC_MAX_ROWS 65536
+int fopd_token_stats_static(const fopd_chunk *chunk /* HOST */, int32_t B, float *lp_s,
+                            float *lp_t, float *kl, float *ratio, double *acc,
+                            int32_t *status, void *stream);
+
+/*
  * Per-sample freshness (Eq. 11), ReLU gate (Eq. 13), alignment ratio and the
  * per-token weight coef_i = w_i / (B |U_i|) that fopd_loss_fwd_bwd applies.
  * A sample with no aligned row, seq_len <= 0 or staleness < 0 is invalid:

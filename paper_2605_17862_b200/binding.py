@@ -19,6 +19,7 @@ FOPD_BF16, FOPD_F32 = 0, 1
 EXPORTS = (
     "fopd_token_stats", "fopd_sample_freshness", "fopd_loss_fwd_bwd", "fopd_loss_finalize",
     "fopd_check_status", "fopd_strerror", "fopd_version", "fopd_step_host", "fopd_step_host_workspace_bytes",
+    "fopd_token_stats_static",
 )
 
 
@@ -65,6 +66,7 @@ def lib() -> ctypes.CDLL:
         L.fopd_strerror.restype = ctypes.c_char_p
         L.fopd_strerror.argtypes = [ctypes.c_int]
         L.fopd_token_stats.argtypes = [ctypes.POINTER(fopd_chunk), i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.fopd_token_stats_static.argtypes = [ctypes.POINTER(fopd_chunk), i32, vp, vp, vp, vp, vp, vp, vp]
         L.fopd_sample_freshness.argtypes = [vp, vp, vp, vp, i32, fopd_params, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.fopd_loss_fwd_bwd.argtypes = [ctypes.POINTER(fopd_chunk), i32, vp, vp, fopd_params, vp, vp, vp, vp]
         L.fopd_loss_finalize.argtypes = [vp, vp, vp, i32, fopd_params, vp, vp, vp]
@@ -140,6 +142,22 @@ def fopd_token_stats(chunk: Chunk, B: int, acc, *, lp_s=None, lp_t=None, kl=None
     _check(lib().fopd_token_stats(ctypes.byref(c), B, _ptr(lp_s), _ptr(lp_t), _ptr(kl), _ptr(ratio),
                                   _ptr(row_ws), _ptr(acc), _ptr(status), _stream(stream)),
            "fopd_token_stats")
+
+
+STATIC_MAX_ROWS = 65536
+
+
+def fopd_token_stats_static(chunk: Chunk, B: int, acc, *, lp_s=None, lp_t=None, kl=None, ratio=None,
+                            status=None, stream=None):
+    """fopd_token_stats without any device allocation: the per-row scratch is a
+    fixed 1 MiB array inside the library (at most STATIC_MAX_ROWS rows per call).
+    For callers that have given all GPU memory to their own allocator or that
+    forbid allocations inside their step loop.  Calls on one device share the
+    scratch, so keep them on one stream."""
+    c = chunk.c_struct()
+    _check(lib().fopd_token_stats_static(ctypes.byref(c), B, _ptr(lp_s), _ptr(lp_t), _ptr(kl), _ptr(ratio),
+                                         _ptr(acc), _ptr(status), _stream(stream)),
+           "fopd_token_stats_static")
 
 
 def fopd_sample_freshness(acc, staleness, seq_len, d_sup, B: int, p: fopd_params, *, coef, f=None,
