@@ -121,6 +121,28 @@ class ClockSampler:
                 "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(value: float, device=None) -> float:
+    """Max of a per-rank scalar over the process group (identity without one)."""
+    import torch
+    import torch.distributed as dist
+
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t[0])
+
+
+def replica_throughput(tokens_per_rank: int, ms_per_step_local: float, device=None):
+    """Replicas-only scaling: every rank processes its own copy of the workload, the
+    job's time is the slowest rank's, its work the sum over ranks."""
+    import torch.distributed as dist
+
+    world = dist.get_world_size() if (dist.is_available() and dist.is_initialized()) else 1
+    ms = max_over_ranks(ms_per_step_local, device)
+    return world * tokens_per_rank / (ms * 1e-3), ms
+
+
 def algorithmic_bytes(wl, active_rows: int):
     """Minimum bytes: statistics sweep reads S and T of aligned rows; the loss
     fwd+bwd reads S and T of differentiated rows once and writes every dlogits row."""
@@ -253,10 +275,6 @@ def main():
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     total_ms = t_begin.elapsed_time(t_end)
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t[0])
     stats_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in events) / len(chunks)
     grad_ms = statistics.mean(e[2].elapsed_time(e[3]) for e in events) / len(chunks)
 
@@ -264,8 +282,7 @@ def main():
     active_rows = int(((coef[np.clip(wl.sample_id, 0, wl.B - 1)] > 0) & (wl.mask > 0)).sum())
     aligned = int(wl.mask.sum())
     stats_bytes, grad_bytes = algorithmic_bytes(wl, active_rows)
-    ms_per_step = total_ms / args.steps
-    value = world * aligned / (ms_per_step * 1e-3)
+    value, ms_per_step = replica_throughput(aligned, total_ms / args.steps, dev)
     peak, peak_src = measured_peak()
     n_launch_chunk = len(chunks)
     kernels_per_step = n_launch_chunk * (2 + (2 if cached else 3)) + 2
@@ -344,11 +361,7 @@ def run_e2e(args, wl, chunks_d, dev, world, aligned):
     for _ in range(args.e2e_steps):
         res = fb.fopd_step_host(hchunks, wl.B, tau, H, None, p, hdl, ws)
     torch.cuda.synchronize()
-    dt = (time.perf_counter() - t0) / args.e2e_steps
-    if world > 1:
-        t = torch.tensor([dt], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        dt = float(t[0])
+    dt = max_over_ranks((time.perf_counter() - t0) / args.e2e_steps, dev)
     logit_bytes = sum(c["student"].numel() * c["student"].element_size() for c in host)
     side = sum(c["tokens"].numel() * 13 for c in host)
     resident = need == fb.fopd_step_host_workspace_bytes(hchunks, wl.B, True)
