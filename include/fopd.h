@@ -79,6 +79,8 @@ typedef enum {
 #define FOPD_DEV_BAD_SAMPLE 2   /* row with sample id outside [0, B)            */
 #define FOPD_DEV_BAD_TAU 4      /* staleness < 0                                */
 #define FOPD_DEV_BAD_LENGTH 8   /* seq_len <= 0 or aligned count > seq_len      */
+#define FOPD_DEV_TIMEOUT 16     /* a bounded in-kernel wait ran out; results of
+                                   that call are not to be trusted               */
 
 /* alpha, beta >= 0 scale the two drift diagnostics (Eq. 11); xi is the gate
  * threshold (Eq. 13); lambda weights the rollout anchor (Eq. 16).  The paper

@@ -3,10 +3,80 @@
 #include <cmath>
 #include <cstdio>
 
+#include "cluster_kernel.cuh"
 #include "host_common.cuh"
 
 using namespace fopd;
 
+
+namespace {
+
+constexpr int kNotApplicable = 1;  // the on-chip kernel cannot take this shape; use the streaming pair
+
+// Fused on-chip forward + backward (cluster_kernel.cuh).  Picks the smallest
+// cluster size whose per-CTA slice of a (student, teacher) row pair fits in
+// shared memory, preferring sizes that leave room for two CTAs per SM.
+template <int DT>
+int launch_fused(const fopd_chunk *chunk, int32_t B, const float *coef, float lambda, void *dlogits,
+                 float *row_ws, int32_t *status, cudaStream_t st) {
+  using E = Elem<DT>;
+  const int64_t nvec = chunk->vocab / E::kPerVec;
+  if (nvec < 1) return kNotApplicable;
+  int dev = 0, max_optin = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&max_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+    return FOPD_ERR_CUDA;
+  const size_t fixed = ((sizeof(ClusterShared) + 127) & ~size_t(127));
+  auto smem_for = [&](int C) { return fixed + 2 * (size_t)((nvec + C - 1) / C) * 16; };
+  const size_t two_per_sm = ((size_t)max_optin + 1024) / 2 - 1024 - 512;  // each CTA also reserves 1 KB
+  int C = 0;
+  for (int cand = 1; cand <= 8 && !C; cand *= 2)
+    if (smem_for(cand) <= two_per_sm) C = cand;
+  for (int cand = 1; cand <= 8 && !C; cand *= 2)
+    if (smem_for(cand) <= (size_t)max_optin) C = cand;
+  if (!C) return kNotApplicable;
+  const size_t smem = smem_for(C);
+  auto kernel = fused_cluster_kernel<DT>;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    return FOPD_ERR_CUDA;
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = C;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.blockDim = dim3(kClusterThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cfg.gridDim = dim3(C);  // placeholder for the occupancy query
+  int max_clusters = 0;
+  if (cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg) != cudaSuccess || max_clusters < 1) {
+    (void)cudaGetLastError();
+    return kNotApplicable;
+  }
+  const int64_t clusters = chunk->n_rows < max_clusters ? chunk->n_rows : max_clusters;
+  cfg.gridDim = dim3((unsigned)(clusters * C));
+  FusedArgs a;
+  a.c = to_dev(chunk);
+  a.B = B;
+  a.coef = coef;
+  a.lambda = lambda;
+  a.dlogits = dlogits;
+  a.row_ws = row_ws;
+  a.status = status;
+  a.slice_vecs = (int)((nvec + C - 1) / C);
+  a.chunk_vecs = kClusterThreads;
+  if ((a.slice_vecs + a.chunk_vecs - 1) / a.chunk_vecs > kMaxChunks) return kNotApplicable;
+  if (cudaLaunchKernelEx(&cfg, kernel, a) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return FOPD_ERR_CUDA;
+  }
+  return FOPD_OK;
+}
+
+}  // namespace
 
 extern "C" {
 
@@ -22,7 +92,7 @@ const char *fopd_strerror(int code) {
     case FOPD_ERR_PARAM: return "alpha/beta must be >= 0 and all parameters finite";
     case FOPD_ERR_CUDA: return "a CUDA runtime call failed";
     case FOPD_ERR_ALIAS: return "dlogits overlaps student or teacher";
-    case FOPD_ERR_DEVICE: return "device status word is non-zero (bad token/sample id, staleness or length)";
+    case FOPD_ERR_DEVICE: return "device status word is non-zero (bad token/sample id, staleness, length or timeout)";
     default: return "unknown fopd status";
   }
 }
@@ -86,15 +156,22 @@ int fopd_loss_fwd_bwd(const fopd_chunk *chunk, int32_t B, const float *coef, con
   const ChunkDev d = to_dev(chunk);
   const float *ws = row_ws;
   float *tmp = nullptr;
+  bool grad_done = false;
   if (!ws) {
-    // No cached statistics: redo the reduction sweep into a temporary workspace.
+    // No cached statistics.  Preferred: the on-chip kernel, which does the reduction sweep
+    // and the gradient sweep from shared memory and leaves the row statistics in tmp.
+    // Shapes it cannot take fall back to the statistics sweep + streaming gradient pair.
     if (cudaMallocAsync(reinterpret_cast<void **>(&tmp), (size_t)chunk->n_rows * 4 * sizeof(float), st) !=
         cudaSuccess)
       return FOPD_ERR_CUDA;
-    rc = launch_stats(chunk, B, nullptr, nullptr, nullptr, nullptr, tmp, status, st, di);
     ws = tmp;
+    rc = chunk->dtype == FOPD_BF16 ? launch_fused<FOPD_BF16>(chunk, B, coef, p.lambda, dlogits, tmp, status, st)
+                                   : launch_fused<FOPD_F32>(chunk, B, coef, p.lambda, dlogits, tmp, status, st);
+    if (rc == FOPD_OK) grad_done = true;
+    else if (rc == kNotApplicable)
+      rc = launch_stats(chunk, B, nullptr, nullptr, nullptr, nullptr, tmp, status, st, di);
   }
-  if (rc == FOPD_OK) {
+  if (rc == FOPD_OK && !grad_done) {
     const int grid = stream_grid(di, chunk->n_rows);
     if (chunk->dtype == FOPD_BF16)
       grad_stream_kernel<FOPD_BF16><<<grid, kStreamThreads, 0, st>>>(d, B, coef, ws, p.lambda, dlogits);

@@ -141,7 +141,7 @@ struct GradRow {
 
 __device__ __forceinline__ GradRow make_grad_row(float4 ws, float coef, float lambda, int32_t y) {
   const float d = ws.w;
-  const float g = lambda * (float)(exp((double)d) * (double)d);
+  const float g = lambda * (expf(d) * d);  // lambda * rho * d, the derivative of lambda * k3
   GradRow r;
   r.e0 = log2f(coef) - ws.x * kLog2e;
   r.K = ws.z + g + (ws.x - ws.y);

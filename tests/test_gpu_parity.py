@@ -197,3 +197,21 @@ def test_host_validation_errors():
     with pytest.raises(fb.FopdError) as e:  # base not 16-byte aligned
         fb.fopd_token_stats(c, wl.B, buf.acc)
     assert e.value.code == -2
+
+
+@pytest.mark.parametrize("V", [40_000, 100_000, 151_936, 300_000, 1_000_000, 40_003])
+def test_standalone_fwd_bwd_across_cluster_sizes(V):
+    """fopd_loss_fwd_bwd without cached statistics keeps each row on chip in a
+    thread-block cluster whose size grows with the vocabulary (1, 2, 4, 8 CTAs);
+    a row too large for eight CTAs falls back to the two streaming kernels."""
+    rng = np.random.RandomState(V % 1000)
+    B, lengths = 3, np.array([9, 17, 14])
+    n = int(lengths.sum())
+    sid = np.repeat(np.arange(B, dtype=np.int32), lengths)
+    mask = (rng.rand(n) > 0.25).astype(np.uint8)
+    wl = synth.Workload("cluster", B, V, torch.bfloat16, n, sid, mask, np.array([0, 1, 2], np.int32),
+                        lengths.astype(np.int32), seed=V % 977)
+    stride = (V + 7) // 8 * 8
+    ch = synth.gen_chunk(wl, 0, DEV, row_block=8, row_stride=stride)
+    out = par.compare([ch], B, wl.tau, wl.H, use_row_ws=False, vocab=V, grad_rows_per_chunk=12)
+    print(V, out)
