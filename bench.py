@@ -295,7 +295,8 @@ def main():
         "config": {
             "workload": wl.name, "rows": wl.n_rows, "aligned_tokens": aligned, "differentiated_rows": active_rows,
             "vocab": wl.V, "samples": wl.B, "logits_dtype": str(wl.dtype).replace("torch.", ""),
-            "chunks": len(chunks), "path": args.path, "tokens_counted": "aligned (mask = 1) rows",
+            "chunks": len(chunks), "path": args.path,
+            "fused_plan": None if cached else fb.fopd_loss_fwd_bwd_plan(wl.dtype, wl.V), "tokens_counted": "aligned (mask = 1) rows",
             "l2": "inputs (2 x %.2f GB) far larger than the 126 MB L2, no flush needed" %
                   (wl.n_rows * wl.V * (2 if wl.dtype == torch.bfloat16 else 4) / 1e9),
             "parallelism": "replicas only" if world > 1 else "1 gpu", "params": P,

@@ -220,6 +220,22 @@ int fopd_loss_fwd_bwd(const fopd_chunk *chunk /* HOST */, int32_t B,
                       void *stream);
 
 /*
+ * Launch shape fopd_loss_fwd_bwd(row_ws = NULL) uses on the current device for
+ * a vocabulary and dtype: CTAs per thread-block cluster (one cluster per row),
+ * slice buffers per CTA (2 = the next row's copies overlap the current row's
+ * sweeps), clusters resident at once and dynamic shared memory per CTA.  All
+ * outputs are HOST pointers and may be NULL.  *cluster_size = 0 means that no
+ * on-chip shape fits (a row pair does not fit in sixteen CTAs' shared memory)
+ * and the call runs the statistics sweep followed by the streaming gradient
+ * sweep instead.  The choice is made once per (device, dtype, vocabulary) with
+ * cudaOccupancyMaxActiveClusters and cached; the environment variables
+ * FOPD_FUSED_CLUSTER and FOPD_FUSED_BUFS, read at that moment, pin it.
+ */
+int fopd_loss_fwd_bwd_plan(int32_t dtype, int64_t vocab, int32_t *cluster_size,
+                           int32_t *slice_buffers, int32_t *resident_clusters,
+                           int32_t *smem_bytes);
+
+/*
  * After the last chunk: per_sample_loss[i] = w_i (l_i + lambda D_roll_i) with
  * l_i, D_roll_i = loss_acc[i] / acc[i].cnt, and loss_out[0] = (1/B) sum_i of
  * it (Eq. 16; Algorithm 1 divides by the minibatch size, gated samples

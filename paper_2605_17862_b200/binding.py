@@ -19,7 +19,7 @@ FOPD_BF16, FOPD_F32 = 0, 1
 EXPORTS = (
     "fopd_token_stats", "fopd_sample_freshness", "fopd_loss_fwd_bwd", "fopd_loss_finalize",
     "fopd_check_status", "fopd_strerror", "fopd_version", "fopd_step_host", "fopd_step_host_workspace_bytes",
-    "fopd_token_stats_static",
+    "fopd_token_stats_static", "fopd_loss_fwd_bwd_plan",
 )
 
 
@@ -69,6 +69,7 @@ def lib() -> ctypes.CDLL:
         L.fopd_token_stats_static.argtypes = [ctypes.POINTER(fopd_chunk), i32, vp, vp, vp, vp, vp, vp, vp]
         L.fopd_sample_freshness.argtypes = [vp, vp, vp, vp, i32, fopd_params, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.fopd_loss_fwd_bwd.argtypes = [ctypes.POINTER(fopd_chunk), i32, vp, vp, fopd_params, vp, vp, vp, vp]
+        L.fopd_loss_fwd_bwd_plan.argtypes = [i32, ctypes.c_int64] + [ctypes.POINTER(ctypes.c_int32)] * 4
         L.fopd_loss_finalize.argtypes = [vp, vp, vp, i32, fopd_params, vp, vp, vp]
         L.fopd_check_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
         L.fopd_step_host_workspace_bytes.restype = ctypes.c_uint64
@@ -176,6 +177,16 @@ def fopd_loss_fwd_bwd(chunk: Chunk, B: int, coef, p: fopd_params, dlogits, loss_
     _check(lib().fopd_loss_fwd_bwd(ctypes.byref(c), B, _ptr(coef), _ptr(row_ws), p, _ptr(dlogits),
                                    _ptr(loss_acc), _ptr(status), _stream(stream)),
            "fopd_loss_fwd_bwd")
+
+
+def fopd_loss_fwd_bwd_plan(dtype: torch.dtype, vocab: int) -> dict:
+    """Launch shape of fopd_loss_fwd_bwd(row_ws=None) on the current device (cluster_size 0:
+    the streaming kernel pair is used instead)."""
+    out = [ctypes.c_int32(0) for _ in range(4)]
+    _check(lib().fopd_loss_fwd_bwd_plan(FOPD_BF16 if dtype == torch.bfloat16 else FOPD_F32, int(vocab),
+                                        *[ctypes.byref(o) for o in out]), "fopd_loss_fwd_bwd_plan")
+    return dict(zip(("cluster_size", "slice_buffers", "resident_clusters", "smem_bytes"),
+                    (int(o.value) for o in out)))
 
 
 def fopd_loss_finalize(loss_acc, acc, w, B: int, p: fopd_params, loss_out, *, per_sample_loss=None,

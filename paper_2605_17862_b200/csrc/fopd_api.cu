@@ -2,6 +2,9 @@
 // caller's stream.  See include/fopd.h for the contract of every entry point.
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
+#include <mutex>
+#include <vector>
 
 #include "cluster_kernel.cuh"
 #include "host_common.cuh"
@@ -13,63 +16,136 @@ namespace {
 
 constexpr int kNotApplicable = 1;  // the on-chip kernel cannot take this shape; use the streaming pair
 
-// Fused on-chip forward + backward (cluster_kernel.cuh).  Picks the smallest
-// cluster size whose per-CTA slice of a (student, teacher) row pair fits in
-// shared memory, preferring sizes that leave room for two CTAs per SM.
+// Launch shape of the on-chip kernel for one (device, dtype, vocabulary): cluster
+// size, shared memory and how many clusters are resident.
+struct FusedPlan {
+  int cluster = 0;     // 0: no shape fits, use the streaming pair
+  int slice_vecs = 0;
+  size_t smem = 0;
+  int max_clusters = 0;
+};
+
 template <int DT>
-int launch_fused(const fopd_chunk *chunk, int32_t B, const float *coef, float lambda, void *dlogits,
-                 float *row_ws, int32_t *status, cudaStream_t st) {
-  using E = Elem<DT>;
-  const int64_t nvec = chunk->vocab / E::kPerVec;
-  if (nvec < 1) return kNotApplicable;
+int set_fused_attributes(int C, size_t smem) {
+  auto kernel = fused_cluster_kernel<DT>;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+      cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, C > 8 ? 1 : 0) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return FOPD_ERR_CUDA;
+  }
+  return FOPD_OK;
+}
+
+static void fused_launch_config(cudaLaunchConfig_t *cfg, cudaLaunchAttribute *attr, int C, size_t smem,
+                                unsigned grid, cudaStream_t st) {
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = C;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  *cfg = cudaLaunchConfig_t{};
+  cfg->blockDim = dim3(kClusterThreads);
+  cfg->gridDim = dim3(grid);
+  cfg->dynamicSmemBytes = smem;
+  cfg->stream = st;
+  cfg->attrs = attr;
+  cfg->numAttrs = 1;
+}
+
+// Picks the cluster size that keeps the most CTAs resident with three slice buffers per
+// CTA (how many clusters of a given size fit depends on how the SMs are grouped), and
+// among equals the smallest.  FOPD_FUSED_CLUSTER in the environment pins the size.
+template <int DT>
+int make_fused_plan(int64_t nvec, FusedPlan *plan) {
   int dev = 0, max_optin = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&max_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
     return FOPD_ERR_CUDA;
   const size_t fixed = ((sizeof(ClusterShared) + 127) & ~size_t(127));
-  auto smem_for = [&](int C) { return fixed + 2 * (size_t)((nvec + C - 1) / C) * 16; };
-  const size_t two_per_sm = ((size_t)max_optin + 1024) / 2 - 1024 - 512;  // each CTA also reserves 1 KB
-  int C = 0;
-  for (int cand = 1; cand <= 8 && !C; cand *= 2)
-    if (smem_for(cand) <= two_per_sm) C = cand;
-  for (int cand = 1; cand <= 8 && !C; cand *= 2)
-    if (smem_for(cand) <= (size_t)max_optin) C = cand;
-  if (!C) return kNotApplicable;
-  const size_t smem = smem_for(C);
-  auto kernel = fused_cluster_kernel<DT>;
-  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-    return FOPD_ERR_CUDA;
-  cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = C;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
-  cfg.blockDim = dim3(kClusterThreads);
-  cfg.dynamicSmemBytes = smem;
-  cfg.stream = st;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  cfg.gridDim = dim3(C);  // placeholder for the occupancy query
-  int max_clusters = 0;
-  if (cudaOccupancyMaxActiveClusters(&max_clusters, kernel, &cfg) != cudaSuccess || max_clusters < 1) {
-    (void)cudaGetLastError();
-    return kNotApplicable;
+  const char *pin_c = getenv("FOPD_FUSED_CLUSTER");
+  FusedPlan best;
+  long best_score = 0;
+  for (int C = 1; C <= kMaxClusterSize; ++C) {
+    if (pin_c && atoi(pin_c) != C) continue;
+    const int64_t slice = (nvec + C - 1) / C;
+    const size_t smem = fixed + (size_t)kSliceBufs * 2 * (size_t)slice * 16;
+    if (smem > (size_t)max_optin || (slice + kClusterThreads - 1) / kClusterThreads > kMaxChunks) continue;
+    int rc = set_fused_attributes<DT>(C, smem);
+    if (rc != FOPD_OK) return rc;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    fused_launch_config(&cfg, attr, C, smem, (unsigned)C, nullptr);
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, fused_cluster_kernel<DT>, &cfg) != cudaSuccess) {
+      (void)cudaGetLastError();
+      n = 0;
+    }
+    const long score = (long)n * C;
+    if (score > best_score) {
+      best_score = score;
+      best.cluster = C;
+      best.slice_vecs = (int)slice;
+      best.smem = smem;
+      best.max_clusters = n;
+    }
   }
-  const int64_t clusters = chunk->n_rows < max_clusters ? chunk->n_rows : max_clusters;
-  cfg.gridDim = dim3((unsigned)(clusters * C));
+  *plan = best;
+  return FOPD_OK;
+}
+
+template <int DT>
+int fused_plan(int64_t nvec, FusedPlan *plan) {
+  struct Entry {
+    int dev;
+    int64_t nvec;
+    FusedPlan plan;
+  };
+  static std::mutex mu;
+  static std::vector<Entry> cache;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FOPD_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(mu);
+  for (const Entry &e : cache)
+    if (e.dev == dev && e.nvec == nvec) {
+      *plan = e.plan;
+      return FOPD_OK;
+    }
+  int rc = make_fused_plan<DT>(nvec, plan);
+  if (rc == FOPD_OK) cache.push_back({dev, nvec, *plan});
+  return rc;
+}
+
+// Fused on-chip forward + backward (cluster_kernel.cuh).  tmp holds [n_rows, 4] row
+// statistics (out) followed by [n_rows] row weights (scratch).
+template <int DT>
+int launch_fused(const fopd_chunk *chunk, int32_t B, const float *coef, float lambda, void *dlogits,
+                 float *tmp, int32_t *status, cudaStream_t st) {
+  using E = Elem<DT>;
+  const int64_t nvec = chunk->vocab / E::kPerVec;
+  if (nvec < 1) return kNotApplicable;
+  FusedPlan plan;
+  int rc = fused_plan<DT>(nvec, &plan);
+  if (rc != FOPD_OK) return rc;
+  if (!plan.cluster || plan.max_clusters < 1) return kNotApplicable;
+  const int C = plan.cluster;
+  // the attributes are per function, and the plan of another vocabulary may have changed them
+  if ((rc = set_fused_attributes<DT>(C, plan.smem)) != FOPD_OK) return rc;
+  float *row_cf = tmp + 4 * chunk->n_rows;
+  const ChunkDev d = to_dev(chunk);
+  row_coef_kernel<<<(unsigned)((chunk->n_rows + 255) / 256), 256, 0, st>>>(d, B, coef, status, row_cf);
+  if ((rc = launch_ok()) != FOPD_OK) return rc;
+  const int64_t clusters = chunk->n_rows < plan.max_clusters ? chunk->n_rows : plan.max_clusters;
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[1];
+  fused_launch_config(&cfg, attr, C, plan.smem, (unsigned)(clusters * C), st);
   FusedArgs a;
-  a.c = to_dev(chunk);
-  a.B = B;
-  a.coef = coef;
+  a.c = d;
   a.lambda = lambda;
   a.dlogits = dlogits;
-  a.row_ws = row_ws;
+  a.row_cf = row_cf;
+  a.row_ws = tmp;
   a.status = status;
-  a.slice_vecs = (int)((nvec + C - 1) / C);
-  a.chunk_vecs = kClusterThreads;
-  if ((a.slice_vecs + a.chunk_vecs - 1) / a.chunk_vecs > kMaxChunks) return kNotApplicable;
-  if (cudaLaunchKernelEx(&cfg, kernel, a) != cudaSuccess) {
+  a.slice_vecs = plan.slice_vecs;
+  if (cudaLaunchKernelEx(&cfg, fused_cluster_kernel<DT>, a) != cudaSuccess) {
     (void)cudaGetLastError();
     return FOPD_ERR_CUDA;
   }
@@ -161,7 +237,7 @@ int fopd_loss_fwd_bwd(const fopd_chunk *chunk, int32_t B, const float *coef, con
     // No cached statistics.  Preferred: the on-chip kernel, which does the reduction sweep
     // and the gradient sweep from shared memory and leaves the row statistics in tmp.
     // Shapes it cannot take fall back to the statistics sweep + streaming gradient pair.
-    if (cudaMallocAsync(reinterpret_cast<void **>(&tmp), (size_t)chunk->n_rows * 4 * sizeof(float), st) !=
+    if (cudaMallocAsync(reinterpret_cast<void **>(&tmp), (size_t)chunk->n_rows * 5 * sizeof(float), st) !=
         cudaSuccess)
       return FOPD_ERR_CUDA;
     ws = tmp;
@@ -185,6 +261,22 @@ int fopd_loss_fwd_bwd(const fopd_chunk *chunk, int32_t B, const float *coef, con
   }
   if (tmp && cudaFreeAsync(tmp, st) != cudaSuccess) rc = FOPD_ERR_CUDA;
   return rc;
+}
+
+int fopd_loss_fwd_bwd_plan(int32_t dtype, int64_t vocab, int32_t *cluster_size, int32_t *slice_buffers,
+                           int32_t *resident_clusters, int32_t *smem_bytes) {
+  if (dtype != FOPD_BF16 && dtype != FOPD_F32) return FOPD_ERR_DTYPE;
+  if (vocab <= 0 || vocab > (int64_t)1 << 30) return FOPD_ERR_SIZE;
+  FusedPlan plan;
+  const int64_t nvec = vocab / (dtype == FOPD_BF16 ? 8 : 4);
+  int rc = FOPD_OK;
+  if (nvec >= 1) rc = dtype == FOPD_BF16 ? fused_plan<FOPD_BF16>(nvec, &plan) : fused_plan<FOPD_F32>(nvec, &plan);
+  if (rc != FOPD_OK) return rc;
+  if (cluster_size) *cluster_size = plan.cluster;
+  if (slice_buffers) *slice_buffers = plan.cluster ? kSliceBufs : 0;
+  if (resident_clusters) *resident_clusters = plan.max_clusters;
+  if (smem_bytes) *smem_bytes = (int32_t)plan.smem;
+  return FOPD_OK;
 }
 
 int fopd_loss_finalize(const double *loss_acc, const double *acc, const float *w, int32_t B,
