@@ -2,42 +2,54 @@
 //
 // A thread-block cluster owns one token row at a time.  Each CTA of the
 // cluster stages its slice of the student and teacher rows in shared memory
-// with bulk asynchronous copies (global -> shared, completion on mbarriers),
-// runs the online max / sum-exp / KL sweep over it, and publishes its partial
-// sums to every CTA of the cluster through distributed shared memory.  Once
-// the cluster barrier has completed every CTA holds the row's normalisers and
-// KL, and the gradient sweep reads the slice back from shared memory and
-// streams dlogits out.  Student and teacher logits are read from HBM once and
-// dlogits written once: 3 * V * e bytes per differentiated row.
+// with bulk asynchronous copies (global -> shared, completion on an mbarrier),
+// runs the online max / sum-exp / KL sweep over it, and sends its partial sums
+// to every CTA of the cluster through distributed shared memory.  Once all
+// partials have landed every CTA holds the row's normalisers and KL, and the
+// gradient sweep reads the slice back from shared memory and streams dlogits
+// out.  Student and teacher logits are read from HBM once and dlogits written
+// once: 3 * V * e bytes per differentiated row.
 //
-// The rows of a cluster move through a three-stage software pipeline over three
-// slice buffers per CTA:
+// Warp 0 of each CTA is a control warp, the other warps compute.  The rows of
+// a cluster move through a software pipeline over three slice buffers per CTA:
 //
-//     step k:   reduction sweep of row k     (buffer k % 3), publish, barrier arrive
-//               gradient sweep of row k - 1  (buffer (k - 1) % 3)
-//               start the copies of row k + 2 into the buffer just freed
-//               barrier wait, row constants of row k
+//   compute warps, step k:  reduction sweep of row k     (buffer k % 3)
+//                           gradient sweep of row k - 1  (buffer (k - 1) % 3)
+//   control warp,  step k:  merge the warps' partials of row k, send them to
+//                           the cluster; start the copies of row k + 2 into
+//                           the buffer of row k - 1 once its gradient sweep is
+//                           done; when all CTAs' partials of row k are here,
+//                           form the row constants for its gradient sweep
 //
 // so the copies of a row are in flight for a whole step before they are
-// needed, and the latency of the cluster exchange of row k is covered by the
-// gradient sweep of row k - 1.  A small kernel run first writes each row's
-// weight coef_i (0 for rows that are not differentiated), which lets the
-// pipeline look rows ahead with independent loads.
+// needed and the cluster exchange of row k is covered by the gradient sweep of
+// row k - 1.  All hand-offs inside a CTA and between CTAs go through mbarriers
+// (no CTA-wide or cluster-wide barrier inside the loop).  A small kernel run
+// first writes each row's weight coef_i (0 for rows that are not
+// differentiated), which lets the pipeline look rows ahead with independent
+// loads.
 //
-// Waits on the copy barriers are bounded; if one ever runs out the CTA records
-// FOPD_DEV_TIMEOUT in the status word and keeps taking part in the cluster
-// barriers (so that no peer is left waiting) until the kernel ends.
+// Every mbarrier wait is bounded; if one runs out the thread records
+// FOPD_DEV_TIMEOUT in the status word, skips its remaining waits and runs to
+// the end of the kernel (the results of that call are void).
 #pragma once
 
-#include "stream_kernels.cuh"
+#include "sweep_math.cuh"
 
 namespace fopd {
 
 constexpr int kClusterThreads = 1024;
+constexpr int kComputeWarps = kClusterThreads / 32 - 1;  // warp 0 is the control warp
+constexpr int kComputeThreads = kComputeWarps * 32;
 constexpr int kMaxClusterSize = 16;
 constexpr int kSliceBufs = 3;
-constexpr int kMaxChunks = 8;                // copy chunks (and mbarriers) per slice buffer
-constexpr uint32_t kSpinLimit = 1u << 22;    // polls of one mbarrier before giving up
+#ifndef FOPD_EXCHANGE_ASYNC
+#define FOPD_EXCHANGE_ASYNC 1
+#endif
+#ifndef FOPD_RELAXED_FREE
+#define FOPD_RELAXED_FREE 1
+#endif
+constexpr long long kWaitCycles = 200000000;  // SM cycles one mbarrier wait may take before giving up (~0.1 s)
 
 // ------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void *p) {
@@ -59,6 +71,33 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Arrival that orders nothing: for "done reading this buffer" signals, issued after the
+// instructions that consumed the data read.
+__device__ __forceinline__ void mbar_arrive_relaxed(uint32_t bar) {
+  asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Stores into another CTA's shared memory that also credit their bytes to an mbarrier of
+// that CTA: the receiver's wait on the barrier covers the data, the sender needs no fence.
+__device__ __forceinline__ void st_async_v4(uint32_t cluster_addr, float a, float b, float c, float d,
+                                            uint32_t cluster_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.f32 [%0], {%1, %2, %3, %4}, [%5];" ::"r"(
+                   cluster_addr),
+               "f"(a), "f"(b), "f"(c), "f"(d), "r"(cluster_bar)
+               : "memory");
+}
+__device__ __forceinline__ void st_async_f32(uint32_t cluster_addr, float a, uint32_t cluster_bar) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];" ::"r"(cluster_addr),
+               "f"(a), "r"(cluster_bar)
+               : "memory");
+}
+// Arrive on an mbarrier of another CTA of the cluster (address from mapa), releasing this
+// thread's earlier distributed-shared-memory stores to whoever acquires the barrier.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -72,13 +111,35 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait: false if the phase did not complete within kSpinLimit polls.
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded waits: false if the phase did not complete within kWaitCycles.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (i > 64) __nanosleep(64);
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > kWaitCycles) return false;
   }
-  return false;
+  return true;
+}
+__device__ __forceinline__ bool mbar_wait_cluster_bounded(uint32_t bar, uint32_t parity) {
+  if (mbar_try_wait_cluster(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait_cluster(bar, parity)) {
+    if (clock64() - t0 > kWaitCycles) return false;
+  }
+  return true;
 }
 __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar) {
   asm volatile(
@@ -105,27 +166,49 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
   return v;
 }
-
-// Cheaper merge for reductions: agree on the maxima first, rescale once, then add.
-__device__ __forceinline__ RowAcc warp_reduce_two_step(RowAcc a) {
-  float Ms = a.ms, Mt = a.mt;
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) {
-    Ms = fmaxf(Ms, __shfl_xor_sync(0xffffffffu, Ms, off));
-    Mt = fmaxf(Mt, __shfl_xor_sync(0xffffffffu, Mt, off));
+// One logit from a staged slice.
+template <int DT>
+__device__ __forceinline__ float lds_logit(uint32_t addr) {
+  float x;
+  if (DT == FOPD_BF16) {
+    unsigned short h;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(h) : "r"(addr));
+    x = __uint_as_float(((uint32_t)h) << 16);
+  } else {
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(x) : "r"(addr));
   }
+  return x;
+}
+__device__ __forceinline__ float warp_max(float x) {
+  float r;
+  asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(x));
+  return r;
+}
+
+// Warp-wide merge of per-lane accumulators: agree on the maxima first (one redux each),
+// rescale once, then add.  The three sums travel in 10 shuffles instead of 15: in the
+// first exchange each lane hands one of (zs, as) to its neighbour and keeps the other.
+// Student and teacher sums are combined in the same order, so equal inputs give equal bits.
+__device__ __forceinline__ RowAcc warp_reduce_two_step(RowAcc a) {
+  const float Ms = warp_max(a.ms), Mt = warp_max(a.mt);
   const float rs = ex2((a.ms - Ms) * kLog2e), rt = ex2((a.mt - Mt) * kLog2e);
-  a.zs *= rs;
-  a.as *= rs;
-  a.zt *= rt;
+  const float zs = a.zs * rs, as = a.as * rs;
+  float zt = a.zt * rt;
+  const bool odd = threadIdx.x & 1;
+  const float give = odd ? zs : as, keep = odd ? as : zs;  // even lanes collect zs, odd lanes as
+  float za = keep + __shfl_xor_sync(0xffffffffu, give, 1);
+  zt += __shfl_xor_sync(0xffffffffu, zt, 1);
+#pragma unroll
+  for (int off = 2; off < 32; off <<= 1) {
+    za += __shfl_xor_sync(0xffffffffu, za, off);
+    zt += __shfl_xor_sync(0xffffffffu, zt, off);
+  }
+  const float other = __shfl_xor_sync(0xffffffffu, za, 1);
+  a.zs = odd ? other : za;
+  a.as = odd ? za : other;
+  a.zt = zt;
   a.ms = Ms;
   a.mt = Mt;
-#pragma unroll
-  for (int off = 16; off > 0; off >>= 1) {
-    a.zs += __shfl_xor_sync(0xffffffffu, a.zs, off);
-    a.as += __shfl_xor_sync(0xffffffffu, a.as, off);
-    a.zt += __shfl_xor_sync(0xffffffffu, a.zt, off);
-  }
   return a;
 }
 
@@ -141,11 +224,20 @@ static __global__ void __launch_bounds__(256)
 }
 
 struct ClusterShared {
-  unsigned long long load_bar[kSliceBufs][kMaxChunks];  // one mbarrier per copy chunk (S and T land on it)
-  RowAcc partial[2][kMaxClusterSize];        // [row parity][source CTA rank], written by peers through DSMEM
+  unsigned long long load_bar[kSliceBufs];   // copies of a slice landed (1 arrival + bytes)
+  unsigned long long free_bar[kSliceBufs];   // gradient sweep of the slice done (one arrival per compute warp)
+  unsigned long long red_bar[2];             // [row parity] warp partials written (one arrival per compute warp)
+  unsigned long long grad_bar[2];            // [row parity] grad_row ready (1 arrival)
+#if FOPD_EXCHANGE_ASYNC
+  unsigned long long xchg_bar[2];            // [row parity] partials of all CTAs here (1 arrival + bytes)
+#else
+  unsigned long long xchg_bar[2];            // [row parity] partials of all CTAs here (one remote arrival per CTA)
+#endif
+  float4 partial4[2][kMaxClusterSize];       // [row parity][source CTA rank] {ms, zs, as, mt}, written by peers
+  float partial_zt[2][kMaxClusterSize];      // [row parity][source CTA rank] zt
   float token_logit[2];                      // [row parity] S[n, y_n], written by the CTA whose slice holds it
-  RowAcc warp_scratch[kClusterThreads / 32];
-  GradRow grad_row[2];                       // [row parity] constants of the gradient sweep, set by thread 0
+  RowAcc warp_scratch[2][32];                // [row parity][compute warp]
+  GradRow grad_row[2];                       // [row parity] constants of the gradient sweep
   int failed;
 };
 
@@ -157,13 +249,26 @@ struct FusedArgs {
   float *row_ws;        // [n_rows,4] out: {lse_s, lse_t, kl, d}; zeros for rows not differentiated
   int32_t *status;
   int slice_vecs;       // 16-byte vectors of a row per CTA (the last CTAs' slices may be shorter or empty)
+#ifdef FOPD_TRACE
+  long long *trace;
+#endif
 };
+
+#ifdef FOPD_TRACE
+#define FOPD_TRACE_AT(id)                                                                \
+  do {                                                                                   \
+    if (a.trace && blockIdx.x == 0 && tid == FOPD_TRACE_TID && k < 64) a.trace[k * 16 + (id)] = clock64(); \
+  } while (0)
+#else
+#define FOPD_TRACE_AT(id) \
+  do {                    \
+  } while (0)
+#endif
 
 template <int DT>
 __global__ void __launch_bounds__(kClusterThreads, 1) fused_cluster_kernel(FusedArgs a) {
   using E = Elem<DT>;
   constexpr int P = E::kPerVec;
-  constexpr int kThreads = kClusterThreads;
   extern __shared__ __align__(128) unsigned char smem_raw[];
   ClusterShared &sh = *reinterpret_cast<ClusterShared *>(smem_raw);
   const uint32_t data_off = (sizeof(ClusterShared) + 127u) & ~127u;
@@ -174,19 +279,28 @@ __global__ void __launch_bounds__(kClusterThreads, 1) fused_cluster_kernel(Fused
   const int64_t n_clusters = gridDim.x / csize, cluster_id = blockIdx.x / csize;
   const ChunkDev &c = a.c;
   const int64_t V = c.vocab, nvec = V / P;
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const bool control = tid < 32;
+  const int ctid = tid - 32;   // index among the compute threads (negative in the control warp)
 
   // This CTA's slice of every row, in vectors.
   const int64_t v_lo = (int64_t)rank * a.slice_vecs;
   const int my_vecs = (int)max((int64_t)0, min((int64_t)a.slice_vecs, nvec - v_lo));
-  const int n_chunks = (my_vecs + kThreads - 1) / kThreads;
   const bool owns_tail = (rank == csize - 1);
-  const int64_t tail_idx = nvec * P + tid;  // scalar tail element handled by the last CTA
+  const int64_t tail_idx = nvec * P + ctid;  // scalar tail element handled by the last CTA's compute threads
+  const bool has_tail = owns_tail && !control && tail_idx < V;
   const int64_t row_bytes = c.stride * E::kBytes;
 
   if (tid == 0) {
-    for (int b = 0; b < kSliceBufs; ++b)
-      for (int k = 0; k < kMaxChunks; ++k) mbar_init(smem_u32(&sh.load_bar[b][k]), 1);
+    for (int b = 0; b < kSliceBufs; ++b) {
+      mbar_init(smem_u32(&sh.load_bar[b]), 1);
+      mbar_init(smem_u32(&sh.free_bar[b]), kComputeWarps);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&sh.red_bar[b]), kComputeWarps);
+      mbar_init(smem_u32(&sh.grad_bar[b]), 1);
+      mbar_init(smem_u32(&sh.xchg_bar[b]), FOPD_EXCHANGE_ASYNC ? 1u : csize);
+    }
     sh.failed = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -194,19 +308,22 @@ __global__ void __launch_bounds__(kClusterThreads, 1) fused_cluster_kernel(Fused
   cluster_arrive();
   cluster_wait();
 
-  // Thread 0 starts the copies of row n's slice into buffer `buf`: one bulk copy per tensor per chunk.
+  // One thread starts the copies of row n's slice into buffer `buf`: one bulk copy per tensor.
   auto issue_row = [&](int64_t n, uint32_t buf) {
+    if (my_vecs == 0) return;
     const char *srow = reinterpret_cast<const char *>(c.student) + n * row_bytes + v_lo * 16;
     const char *trow = reinterpret_cast<const char *>(c.teacher) + n * row_bytes + v_lo * 16;
     const uint32_t s_base = data_base + buf * 2u * slice_bytes, t_base = s_base + slice_bytes;
-    for (int k = 0; k < n_chunks; ++k) {
-      const int v0 = k * kThreads;
-      const uint32_t bytes = (uint32_t)min(kThreads, my_vecs - v0) * 16u;
-      const uint32_t bar = smem_u32(&sh.load_bar[buf][k]);
-      mbar_expect_tx(bar, 2u * bytes);
-      bulk_load(s_base + (uint32_t)v0 * 16u, srow + (int64_t)v0 * 16, bytes, bar);
-      bulk_load(t_base + (uint32_t)v0 * 16u, trow + (int64_t)v0 * 16, bytes, bar);
-    }
+    const uint32_t bytes = (uint32_t)my_vecs * 16u, bar = smem_u32(&sh.load_bar[buf]);
+    mbar_expect_tx(bar, 2u * bytes);
+    bulk_load(s_base, srow, bytes, bar);
+    bulk_load(t_base, trow, bytes, bar);
+  };
+  // After one wait has run out the rest are skipped: the results are void anyway and the
+  // kernel must end soon.
+  bool ok = true;
+  auto wait_on = [&](unsigned long long *bar, uint32_t parity) {
+    if (ok) ok = mbar_wait_bounded(smem_u32(bar), parity);
   };
 
   // ---- scan over this cluster's rows, row weights fetched three rows ahead
@@ -230,8 +347,9 @@ __global__ void __launch_bounds__(kClusterThreads, 1) fused_cluster_kernel(Fused
       char *orow = reinterpret_cast<char *>(a.dlogits) + n * row_bytes;
       uint4 *o4 = reinterpret_cast<uint4 *>(orow) + v_lo;
       const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-      for (int i = tid; i < my_vecs; i += kThreads) st_stream(o4 + i, z);
-      if (owns_tail && tail_idx < V) E::store1(orow, tail_idx, 0.f);
+      if (!control)
+        for (int i = ctid; i < my_vecs; i += kComputeThreads) st_stream(o4 + i, z);
+      if (has_tail) E::store1(orow, tail_idx, 0.f);
       if (rank == 0 && tid == 0) reinterpret_cast<float4 *>(a.row_ws)[n] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     cf_out = 0.f;
@@ -248,42 +366,24 @@ __global__ void __launch_bounds__(kClusterThreads, 1) fused_cluster_kernel(Fused
   if (row_l >= 0 && tid == 0) issue_row(row_l, 1);
 
   for (uint32_t k = 0; row_r >= 0 || row_g >= 0; ++k) {
-    // side inputs of row k that warp 0 needs after the sweep: fetched now, used late
-    int32_t y = 0;
-    float b = 0.f;
-    if (row_r >= 0 && tid < 32) {
-      y = c.tokens[row_r];
-      b = c.behav[row_r];
-    }
-    // ---- reduction sweep of row k
-    if (row_r >= 0) {
-      const uint32_t buf = k % kSliceBufs, parity = (k / kSliceBufs) & 1u, slot = k & 1u;
-      const uint32_t s_base = data_base + buf * 2u * slice_bytes, t_base = s_base + slice_bytes;
-      const char *srow = reinterpret_cast<const char *>(c.student) + row_r * row_bytes;
-      const char *trow = reinterpret_cast<const char *>(c.teacher) + row_r * row_bytes;
-
-      RowAcc acc;
-      acc.init();
-      bool ok = true;
-      for (int kc = 0; kc < n_chunks; ++kc) {
-        ok = mbar_wait_bounded(smem_u32(&sh.load_bar[buf][kc]), parity) && ok;
-        const int i = kc * kThreads + tid;
-        if (i < my_vecs) {
-          float s[P], t[P];
-          E::unpack(lds128(s_base + (uint32_t)i * 16u), s);
-          E::unpack(lds128(t_base + (uint32_t)i * 16u), t);
-          acc.add<P>(s, t);
-        }
-      }
-      if (!ok) sh.failed = 1;
-      if (owns_tail && tail_idx < V) acc.add1(E::load1(srow, tail_idx), E::load1(trow, tail_idx));
-
-      // CTA partial (and the stored token's logit) published to every CTA through DSMEM
-      acc = warp_reduce_two_step(acc);
-      if ((tid & 31) == 0) sh.warp_scratch[tid >> 5] = acc;
-      __syncthreads();  // also publishes grad_row of row k - 1 to the gradient sweep below
-      if (tid < 32) {
-        RowAcc r = sh.warp_scratch[tid];
+    FOPD_TRACE_AT(0);
+    const uint32_t slot = k & 1u, par2 = (k >> 1) & 1u;
+    const uint32_t buf_r = k % kSliceBufs, buf_g = (k + kSliceBufs - 1) % kSliceBufs;
+    float cf_n = 0.f;
+    int64_t row_n = -1;
+    if (control) {
+      // =================================================== control warp
+      int32_t y = 0;
+      float b = 0.f;
+      if (row_r >= 0) {
+        y = c.tokens[row_r];   // used after the waits below
+        b = c.behav[row_r];
+        // CTA partial: every compute warp has written its own
+        wait_on(&sh.red_bar[slot], par2);
+        FOPD_TRACE_AT(1);
+        RowAcc r;
+        r.init();
+        if (lane < kComputeWarps) r = sh.warp_scratch[slot][lane];
         r = warp_reduce_two_step(r);
         // which CTA holds S[n, y]: the slice that contains its vector, or the last CTA for the scalar tail
         const int64_t yv = y / P;
@@ -292,73 +392,133 @@ __global__ void __launch_bounds__(kClusterThreads, 1) fused_cluster_kernel(Fused
         float sy = 0.f;
         if (mine) {
           if (in_body) {
-            const uint32_t addr = s_base + (uint32_t)((int64_t)y - v_lo * P) * E::kBytes;
-            if (DT == FOPD_BF16) {
-              unsigned short h;
-              asm volatile("ld.shared.u16 %0, [%1];" : "=h"(h) : "r"(addr));
-              sy = __uint_as_float(((uint32_t)h) << 16);
-            } else {
-              asm volatile("ld.shared.f32 %0, [%1];" : "=f"(sy) : "r"(addr));
-            }
+            wait_on(&sh.load_bar[buf_r], (k / kSliceBufs) & 1u);
+            sy = lds_logit<DT>(data_base + buf_r * 2u * slice_bytes + (uint32_t)((int64_t)y - v_lo * P) * E::kBytes);
           } else {
-            sy = E::load1(srow, y);
+            sy = E::load1(reinterpret_cast<const char *>(c.student) + row_r * row_bytes, y);
           }
         }
-        if (tid < (int)csize) {
-          const uint32_t dst = map_to_cta(smem_u32(&sh.partial[slot][rank]), (uint32_t)tid);
+        // lane j sends this CTA's partial (and the token's logit) to CTA j
+#if FOPD_EXCHANGE_ASYNC
+        // every CTA (this one included) receives 20 bytes from each CTA and 4 from the token's owner
+        if (lane == 0) mbar_expect_tx(smem_u32(&sh.xchg_bar[slot]), csize * 20u + 4u);
+        if (lane < (int)csize) {
+          const uint32_t bar = map_to_cta(smem_u32(&sh.xchg_bar[slot]), (uint32_t)lane);
+          st_async_v4(map_to_cta(smem_u32(&sh.partial4[slot][rank]), (uint32_t)lane), r.ms, r.zs, r.as, r.mt, bar);
+          st_async_f32(map_to_cta(smem_u32(&sh.partial_zt[slot][rank]), (uint32_t)lane), r.zt, bar);
+          if (mine) st_async_f32(map_to_cta(smem_u32(&sh.token_logit[slot]), (uint32_t)lane), sy, bar);
+        }
+        FOPD_TRACE_AT(2);
+#else
+        if (lane < (int)csize) {
+          const uint32_t dst = map_to_cta(smem_u32(&sh.partial4[slot][rank]), (uint32_t)lane);
           st_cluster_f32(dst + 0, r.ms);
           st_cluster_f32(dst + 4, r.zs);
           st_cluster_f32(dst + 8, r.as);
           st_cluster_f32(dst + 12, r.mt);
-          st_cluster_f32(dst + 16, r.zt);
-          if (mine) st_cluster_f32(map_to_cta(smem_u32(&sh.token_logit[slot]), (uint32_t)tid), sy);
+          st_cluster_f32(map_to_cta(smem_u32(&sh.partial_zt[slot][rank]), (uint32_t)lane), r.zt);
+          if (mine) st_cluster_f32(map_to_cta(smem_u32(&sh.token_logit[slot]), (uint32_t)lane), sy);
+          FOPD_TRACE_AT(2);
+          mbar_arrive_remote(map_to_cta(smem_u32(&sh.xchg_bar[slot]), (uint32_t)lane));
         }
+#endif
+        FOPD_TRACE_AT(3);
       }
-      cluster_arrive();
-    } else {
-      __syncthreads();  // publishes grad_row of the last row
-    }
-
-    // ---- gradient sweep of row k - 1 from its resident slice, streamed out
-    if (row_g >= 0) {
-      const uint32_t buf = (k + kSliceBufs - 1) % kSliceBufs;
-      const uint32_t s_base = data_base + buf * 2u * slice_bytes, t_base = s_base + slice_bytes;
-      const GradRow gr = sh.grad_row[(k + 1) & 1u];
-      char *orow = reinterpret_cast<char *>(a.dlogits) + row_g * row_bytes;
-      uint4 *o4 = reinterpret_cast<uint4 *>(orow) + v_lo;
-      for (int i = tid; i < my_vecs; i += kThreads) {
-        const uint4 sv = lds128(s_base + (uint32_t)i * 16u), tv = lds128(t_base + (uint32_t)i * 16u);
-        st_stream(o4 + i, grad_vec<DT>(sv, tv, gr, (v_lo + i) * P));
+      // look ahead: row k + 2 goes into the buffer of row k - 1 once its gradient sweep is done
+      row_n = row_l >= 0 ? next_row(cf_n) : -1;
+      if (row_n >= 0) {
+        if (row_g >= 0) wait_on(&sh.free_bar[buf_g], ((k - 1) / kSliceBufs) & 1u);
+        FOPD_TRACE_AT(4);
+        if (lane == 0) issue_row(row_n, (k + 2) % kSliceBufs);
+        FOPD_TRACE_AT(5);
       }
-      if (owns_tail && tail_idx < V) {
-        const char *srow = reinterpret_cast<const char *>(c.student) + row_g * row_bytes;
-        const char *trow = reinterpret_cast<const char *>(c.teacher) + row_g * row_bytes;
-        const float s = E::load1(srow, tail_idx), t = E::load1(trow, tail_idx);
-        float o = ex2(fmaf(s, kLog2e, gr.e0)) * ((s - t) - gr.K);
-        if (tail_idx == gr.y) o += gr.cg;
-        E::store1(orow, tail_idx, o);
-      }
-    }
-    __syncthreads();  // the buffer of row k - 1 is free
-
-    // ---- look ahead: row k + 2 goes into the buffer just freed ((k + 2) % 3 == (k - 1) % 3)
-    float cf_n = 0.f;
-    const int64_t row_n = row_l >= 0 ? next_row(cf_n) : -1;
-    if (row_n >= 0 && tid == 0) issue_row(row_n, (k + 2) % kSliceBufs);
-
-    // ---- finish the exchange of row k: row constants, identical in every CTA
-    if (row_r >= 0) {
-      cluster_wait();
-      if (tid == 0) {
-        const uint32_t slot = k & 1u;
-        RowAcc r = sh.partial[slot][0];
-        for (uint32_t j = 1; j < csize; ++j) r.merge(sh.partial[slot][j]);
+      // finish the exchange of row k: row constants, identical in every CTA
+      if (row_r >= 0) {
+        if (ok) ok = mbar_wait_cluster_bounded(smem_u32(&sh.xchg_bar[slot]), par2);
+        FOPD_TRACE_AT(6);
+        RowAcc r;
+        r.init();
+        if (lane < (int)csize) {
+          const float4 p4 = sh.partial4[slot][lane];
+          r.ms = p4.x;
+          r.zs = p4.y;
+          r.as = p4.z;
+          r.mt = p4.w;
+          r.zt = sh.partial_zt[slot][lane];
+        }
+        r = warp_reduce_two_step(r);
         const float ls = r.ms + logf(r.zs), lt = r.mt + logf(r.zt);
         const float kl = r.as / r.zs - (ls - lt);
         const float d = (sh.token_logit[slot] - ls) - b;
-        sh.grad_row[slot] = make_grad_row(make_float4(ls, lt, kl, d), cf_r, a.lambda, y);
-        if (rank == 0) reinterpret_cast<float4 *>(a.row_ws)[row_r] = make_float4(ls, lt, kl, d);
+        if (lane == 0) {
+          sh.grad_row[slot] = make_grad_row(make_float4(ls, lt, kl, d), cf_r, a.lambda, y);
+          mbar_arrive(smem_u32(&sh.grad_bar[slot]));
+          if (rank == 0) reinterpret_cast<float4 *>(a.row_ws)[row_r] = make_float4(ls, lt, kl, d);
+        }
+        FOPD_TRACE_AT(7);
       }
+    } else {
+      // =================================================== compute warps
+      if (row_r >= 0) {
+        const uint32_t s_base = data_base + buf_r * 2u * slice_bytes, t_base = s_base + slice_bytes;
+        if (my_vecs > 0) wait_on(&sh.load_bar[buf_r], (k / kSliceBufs) & 1u);
+        FOPD_TRACE_AT(1);
+        SweepAcc<DT> sweep;
+        sweep.init();
+        for (int i = ctid; i < my_vecs; i += kComputeThreads)
+          sweep.add(lds128(s_base + (uint32_t)i * 16u), lds128(t_base + (uint32_t)i * 16u));
+        if (has_tail) {
+          const char *srow = reinterpret_cast<const char *>(c.student) + row_r * row_bytes;
+          const char *trow = reinterpret_cast<const char *>(c.teacher) + row_r * row_bytes;
+          sweep.add1(E::load1(srow, tail_idx), E::load1(trow, tail_idx));
+        }
+        FOPD_TRACE_AT(2);
+        const RowAcc acc = warp_reduce_two_step(sweep.fold());
+        if (lane == 0) {
+          sh.warp_scratch[slot][(tid >> 5) - 1] = acc;
+          mbar_arrive(smem_u32(&sh.red_bar[slot]));
+        }
+        FOPD_TRACE_AT(3);
+      }
+      if (row_g >= 0) {
+        const uint32_t s_base = data_base + buf_g * 2u * slice_bytes, t_base = s_base + slice_bytes;
+        wait_on(&sh.grad_bar[slot ^ 1u], ((k - 1) >> 1) & 1u);
+        FOPD_TRACE_AT(5);
+        const GradRow gr = sh.grad_row[slot ^ 1u];
+        char *orow = reinterpret_cast<char *>(a.dlogits) + row_g * row_bytes;
+        uint4 *o4 = reinterpret_cast<uint4 *>(orow) + v_lo;
+        for (int i = ctid; i < my_vecs; i += kComputeThreads) {
+          const uint4 sv = lds128(s_base + (uint32_t)i * 16u), tv = lds128(t_base + (uint32_t)i * 16u);
+          st_stream(o4 + i, grad_body<DT>(sv, tv, gr));
+        }
+        {
+          // the stored token's element gets its extra term from the thread that wrote its vector
+          // (same thread, so the two stores to that address stay in order)
+          const int64_t yv = gr.y / P - v_lo;
+          if (yv >= 0 && yv < my_vecs && (int)(yv % kComputeThreads) == ctid) {
+            const uint32_t off = (uint32_t)((int64_t)gr.y - v_lo * P) * E::kBytes;
+            const float s = lds_logit<DT>(s_base + off), t = lds_logit<DT>(t_base + off);
+            E::store1(orow, gr.y, fmaf(ex2(fmaf(s, kLog2e, gr.e0)), (s - t) - gr.K, gr.cg));
+          }
+        }
+        if (has_tail) {
+          const char *srow = reinterpret_cast<const char *>(c.student) + row_g * row_bytes;
+          const char *trow = reinterpret_cast<const char *>(c.teacher) + row_g * row_bytes;
+          const float s = E::load1(srow, tail_idx), t = E::load1(trow, tail_idx);
+          float o = ex2(fmaf(s, kLog2e, gr.e0)) * ((s - t) - gr.K);
+          if (tail_idx == gr.y) o += gr.cg;
+          E::store1(orow, tail_idx, o);
+        }
+        FOPD_TRACE_AT(6);
+        __syncwarp();
+#if FOPD_RELAXED_FREE
+        if (lane == 0) mbar_arrive_relaxed(smem_u32(&sh.free_bar[buf_g]));
+#else
+        if (lane == 0) mbar_arrive(smem_u32(&sh.free_bar[buf_g]));
+#endif
+      }
+      row_n = row_l >= 0 ? next_row(cf_n) : -1;
+      FOPD_TRACE_AT(7);
     }
     row_g = row_r;
     row_r = row_l;
@@ -367,6 +527,8 @@ __global__ void __launch_bounds__(kClusterThreads, 1) fused_cluster_kernel(Fused
     cf_l = cf_n;
   }
 
+  if (!ok) sh.failed = 1;
+  __syncthreads();
   if (tid == 0 && sh.failed && a.status) atomicOr(a.status, FOPD_DEV_TIMEOUT);
   // No CTA may exit while a peer can still write into its shared memory.
   cluster_arrive();

@@ -68,7 +68,7 @@ int make_fused_plan(int64_t nvec, FusedPlan *plan) {
     if (pin_c && atoi(pin_c) != C) continue;
     const int64_t slice = (nvec + C - 1) / C;
     const size_t smem = fixed + (size_t)kSliceBufs * 2 * (size_t)slice * 16;
-    if (smem > (size_t)max_optin || (slice + kClusterThreads - 1) / kClusterThreads > kMaxChunks) continue;
+    if (smem > (size_t)max_optin || slice * 32 >= (1 << 20)) continue;  // one copy barrier counts < 2^20 bytes
     int rc = set_fused_attributes<DT>(C, smem);
     if (rc != FOPD_OK) return rc;
     cudaLaunchConfig_t cfg;
