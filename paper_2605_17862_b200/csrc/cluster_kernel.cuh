@@ -124,22 +124,27 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
       : "memory");
   return ok != 0;
 }
-// Bounded waits: false if the phase did not complete within kWaitCycles.
+// Bounded waits: false if the phase did not complete within kWaitCycles.  try_wait itself
+// parks the thread for a while, so the loop is kept to the poll and a branch; the clock is
+// read once per kPollsPerClock polls.
+constexpr int kPollsPerClock = 256;
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > kWaitCycles) return false;
-  }
-  return true;
+  do {
+    for (int i = 0; i < kPollsPerClock; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+  } while (clock64() - t0 <= kWaitCycles);
+  return false;
 }
 __device__ __forceinline__ bool mbar_wait_cluster_bounded(uint32_t bar, uint32_t parity) {
   if (mbar_try_wait_cluster(bar, parity)) return true;
   const long long t0 = clock64();
-  while (!mbar_try_wait_cluster(bar, parity)) {
-    if (clock64() - t0 > kWaitCycles) return false;
-  }
-  return true;
+  do {
+    for (int i = 0; i < kPollsPerClock; ++i)
+      if (mbar_try_wait_cluster(bar, parity)) return true;
+  } while (clock64() - t0 <= kWaitCycles);
+  return false;
 }
 __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar) {
   asm volatile(

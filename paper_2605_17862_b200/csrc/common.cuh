@@ -20,6 +20,22 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// max of three (one instruction on sm_100a)
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+template <int N>
+__device__ __forceinline__ float max_of(const float (&x)[N]) {
+  if (N == 8) return fmaxf(max3(x[0], x[1], x[2]), max3(x[3], x[4], max3(x[5], x[6], x[7 % N])));
+  if (N == 4) return fmaxf(x[0], max3(x[1], x[2 % N], x[3 % N]));
+  float v = x[0];
+#pragma unroll
+  for (int i = 1; i < N; ++i) v = fmaxf(v, x[i]);
+  return v;
+}
+
 // Streaming (read-once) 16-byte global load.
 __device__ __forceinline__ uint4 ld_stream(const void *p) {
   uint4 v;
@@ -103,12 +119,7 @@ struct RowAcc {
   // Fold N (s, t) pairs in; the maxima move only when a vector beats them.
   template <int N>
   __device__ __forceinline__ void add(const float (&s)[N], const float (&t)[N]) {
-    float vs = s[0], vt = t[0];
-#pragma unroll
-    for (int i = 1; i < N; ++i) {
-      vs = fmaxf(vs, s[i]);
-      vt = fmaxf(vt, t[i]);
-    }
+    const float vs = max_of<N>(s), vt = max_of<N>(t);
     if (vs > ms) {
       const float r = ex2((ms - vs) * kLog2e);
       zs *= r;

@@ -43,18 +43,14 @@ __device__ __forceinline__ bool row_is_aligned(const ChunkDev &c, int64_t n, int
 // Turns the finished accumulators of a row into the quantities of Sec. 4.1 /
 // Eq. 10 / Eq. 12 and writes the per-row outputs.  Called by one thread.
 template <int DT>
-__device__ __forceinline__ void finish_row(const ChunkDev &c, int64_t n, const RowAcc &r, float *lp_s,
+__device__ __forceinline__ void finish_row(int64_t n, const RowAcc &r, float sy, float ty, float b, float *lp_s,
                                            float *lp_t, float *kl_out, float *ratio, float *row_ws) {
-  using E = Elem<DT>;
   // log of the partition sums in full precision (logf, not the fast intrinsic)
   const float ls = r.ms + logf(r.zs);
   const float lt = r.mt + logf(r.zt);
   const float kl = r.as / r.zs - (ls - lt);
-  const int32_t y = c.tokens[n];
-  const float sy = E::load1(c.student, n * c.stride + y);
-  const float ty = E::load1(c.teacher, n * c.stride + y);
   const float lps = sy - ls, lpt = ty - lt;
-  const float d = lps - c.behav[n];
+  const float d = lps - b;
   if (lp_s) lp_s[n] = lps;
   if (lp_t) lp_t[n] = lpt;
   if (kl_out) kl_out[n] = kl;
@@ -114,19 +110,49 @@ __global__ void __launch_bounds__(kStreamThreads, 2)
     token_stats_kernel(ChunkDev c, int32_t B, float *lp_s, float *lp_t, float *kl, float *ratio,
                        float *row_ws, int32_t *status) {
   using E = Elem<DT>;
-  __shared__ RowAcc scratch[kStreamThreads / 32];
-  for (int64_t n = blockIdx.x; n < c.n_rows; n += gridDim.x) {
-    const bool ok = row_is_aligned(c, n, B, status, threadIdx.x == 0);
-    if (!ok) {
+  __shared__ RowAcc scratch[2][kStreamThreads / 32];  // alternating per row: no barrier after the row's finish
+  const int64_t step = gridDim.x;
+  // id, token and mask of the next row are fetched while this row is swept
+  auto side = [&](int64_t n, int32_t &sid, int32_t &y, uint32_t &m) {
+    const bool in = n < c.n_rows;
+    sid = in ? c.sid[n] : 0;
+    y = in ? c.tokens[n] : 0;
+    m = in ? c.mask[n] : 0u;
+  };
+  int64_t n = blockIdx.x;
+  int32_t sid_n, y_n;
+  uint32_t m_n;
+  side(n, sid_n, y_n, m_n);
+  for (int par = 0; n < c.n_rows; n += step) {
+    const int32_t sid = sid_n, y = y_n;
+    const uint32_t m = m_n;
+    side(n + step, sid_n, y_n, m_n);
+    bool ok = true;
+    if (sid < 0 || sid >= B) {
+      if (threadIdx.x == 0 && status) atomicOr(status, FOPD_DEV_BAD_SAMPLE);
+      ok = false;
+    }
+    if (m != 0u && (y < 0 || y >= c.vocab)) {
+      if (threadIdx.x == 0 && status) atomicOr(status, FOPD_DEV_BAD_TOKEN);
+      ok = false;
+    }
+    if (!ok || m == 0u) {
       if (threadIdx.x == 0) zero_row_outputs(n, lp_s, lp_t, kl, ratio, row_ws);
       continue;
+    }
+    // gathers of the stored token and its behaviour log-prob: issued now, used after the sweep
+    float sy = 0.f, ty = 0.f, b = 0.f;
+    if (threadIdx.x == 0) {
+      sy = E::load1(c.student, n * c.stride + y);
+      ty = E::load1(c.teacher, n * c.stride + y);
+      b = c.behav[n];
     }
     const char *srow = reinterpret_cast<const char *>(c.student) + n * c.stride * E::kBytes;
     const char *trow = reinterpret_cast<const char *>(c.teacher) + n * c.stride * E::kBytes;
     RowAcc acc = sweep_row_global<DT, kStreamThreads>(srow, trow, c.vocab);
-    acc = block_reduce<kStreamThreads>(acc, scratch);
-    if (threadIdx.x == 0) finish_row<DT>(c, n, acc, lp_s, lp_t, kl, ratio, row_ws);
-    __syncthreads();  // scratch is reused by the next row
+    acc = block_reduce<kStreamThreads>(acc, scratch[par]);
+    if (threadIdx.x == 0) finish_row<DT>(n, acc, sy, ty, b, lp_s, lp_t, kl, ratio, row_ws);
+    par ^= 1;
   }
 }
 
@@ -150,25 +176,17 @@ __device__ __forceinline__ GradRow make_grad_row(float4 ws, float coef, float la
   return r;
 }
 
+// Gradient of one vector without the stored token's extra term (added afterwards by
+// the thread that wrote the token's vector).
 template <int DT>
-__device__ __forceinline__ uint4 grad_vec(const uint4 &sv, const uint4 &tv, const GradRow &r,
-                                          int64_t v0) {
+__device__ __forceinline__ uint4 grad_vec(const uint4 &sv, const uint4 &tv, const GradRow &r) {
   using E = Elem<DT>;
   constexpr int P = E::kPerVec;
   float s[P], t[P], o[P];
   E::unpack(sv, s);
   E::unpack(tv, t);
 #pragma unroll
-  for (int i = 0; i < P; ++i) {
-    const float cp = ex2(fmaf(s[i], kLog2e, r.e0));
-    o[i] = cp * ((s[i] - t[i]) - r.K);
-  }
-  const int64_t off = (int64_t)r.y - v0;
-  if (off >= 0 && off < P) {
-#pragma unroll
-    for (int i = 0; i < P; ++i)
-      if (i == off) o[i] += r.cg;
-  }
+  for (int i = 0; i < P; ++i) o[i] = ex2(fmaf(s[i], kLog2e, r.e0)) * ((s[i] - t[i]) - r.K);
   return E::pack(o);
 }
 
@@ -181,11 +199,40 @@ __global__ void __launch_bounds__(kStreamThreads, 2)
   constexpr int P = E::kPerVec;
   constexpr int kThreads = kStreamThreads;
   const int64_t V = c.vocab, nvec = V / P;
-  for (int64_t n = blockIdx.x; n < c.n_rows; n += gridDim.x) {
+  // The side inputs of a row hang off two dependent loads (sample id -> coef), each a trip to
+  // L2 under load.  They are fetched ahead in two stages so that no row waits for them:
+  // stage A (two rows ahead) loads id, mask and token, stage B (one row ahead) uses the id
+  // to load coef and the cached statistics.
+  const int64_t step = gridDim.x;
+  auto in_range = [&](int64_t n) { return n < c.n_rows; };
+  auto stage_a = [&](int64_t n, int32_t &sid, int32_t &y, uint32_t &m) {
+    sid = in_range(n) ? c.sid[n] : -1;
+    y = in_range(n) ? c.tokens[n] : 0;
+    m = in_range(n) ? c.mask[n] : 0u;
+  };
+  auto stage_b = [&](int64_t n, int32_t sid, int32_t y, uint32_t m, float &cf, float4 &ws) {
+    const bool ok = m != 0u && sid >= 0 && sid < B && y >= 0 && y < V;
+    cf = ok ? coef[sid] : 0.f;
+    ws = ok ? reinterpret_cast<const float4 *>(row_ws)[n] : make_float4(0.f, 0.f, 0.f, 0.f);
+  };
+  int64_t n = blockIdx.x;
+  int32_t sid_a, y_a, y_b;
+  uint32_t m_a;
+  float cf_b;
+  float4 ws_b;
+  stage_a(n, sid_a, y_a, m_a);
+  stage_b(n, sid_a, y_a, m_a, cf_b, ws_b);
+  y_b = y_a;
+  stage_a(n + step, sid_a, y_a, m_a);
+  for (; n < c.n_rows; n += step) {
+    const float cf = cf_b;
+    const float4 ws = ws_b;
+    const int32_t y = y_b;
+    stage_b(n + step, sid_a, y_a, m_a, cf_b, ws_b);   // in flight while this row is swept
+    y_b = y_a;
+    stage_a(n + 2 * step, sid_a, y_a, m_a);
     char *orow = reinterpret_cast<char *>(dlogits) + n * c.stride * E::kBytes;
     uint4 *o4 = reinterpret_cast<uint4 *>(orow);
-    float cf = 0.f;
-    if (row_is_aligned(c, n, B, nullptr, false)) cf = coef[c.sid[n]];
     if (!(cf > 0.f)) {  // masked, padded, bad id, gated or invalid sample: +0
       const uint4 z = make_uint4(0u, 0u, 0u, 0u);
       for (int64_t i = threadIdx.x; i < nvec; i += kThreads) st_stream(o4 + i, z);
@@ -193,7 +240,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2)
       if (tail < V) E::store1(orow, tail, 0.f);
       continue;
     }
-    const GradRow r = make_grad_row(reinterpret_cast<const float4 *>(row_ws)[n], cf, lambda, c.tokens[n]);
+    const GradRow r = make_grad_row(ws, cf, lambda, y);
     const char *srow = reinterpret_cast<const char *>(c.student) + n * c.stride * E::kBytes;
     const char *trow = reinterpret_cast<const char *>(c.teacher) + n * c.stride * E::kBytes;
     const uint4 *s4 = reinterpret_cast<const uint4 *>(srow);
@@ -208,10 +255,17 @@ __global__ void __launch_bounds__(kStreamThreads, 2)
       }
 #pragma unroll
       for (int u = 0; u < kUnroll; ++u)
-        st_stream(o4 + i + u * kThreads, grad_vec<DT>(a[u], b[u], r, (i + u * kThreads) * P));
+        st_stream(o4 + i + u * kThreads, grad_vec<DT>(a[u], b[u], r));
     }
     for (; i < nvec; i += kThreads)
-      st_stream(o4 + i, grad_vec<DT>(ld_stream(s4 + i), ld_stream(t4 + i), r, i * P));
+      st_stream(o4 + i, grad_vec<DT>(ld_stream(s4 + i), ld_stream(t4 + i), r));
+    // the stored token's element: rewritten with its extra term by the thread that stored its
+    // vector (one thread, so the two stores to that address stay in order)
+    const int64_t yv = r.y / P;
+    if (yv < nvec && (int)(yv % kThreads) == (int)threadIdx.x) {
+      const float s = E::load1(srow, r.y), t = E::load1(trow, r.y);
+      E::store1(orow, r.y, fmaf(ex2(fmaf(s, kLog2e, r.e0)), (s - t) - r.K, r.cg));
+    }
     const int64_t tail = nvec * P + threadIdx.x;
     if (tail < V) {
       const float s = E::load1(srow, tail), t = E::load1(trow, tail);

@@ -49,12 +49,6 @@ __device__ __forceinline__ f32x2 ex2_2(f32x2 a) {
   unpack2(a, lo, hi);
   return pack2(ex2(lo), ex2(hi));
 }
-__device__ __forceinline__ float max3(float a, float b, float c) {
-  float d;
-  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-  return d;
-}
-
 // One 16-byte vector as fp32 pairs (adjacent logits share a pair).
 template <int DT>
 struct Pairs;
