@@ -248,11 +248,11 @@ int fopd_loss_fwd_bwd(const fopd_chunk *chunk, int32_t B, const float *coef, con
       rc = launch_stats(chunk, B, nullptr, nullptr, nullptr, nullptr, tmp, status, st, di);
   }
   if (rc == FOPD_OK && !grad_done) {
-    const int grid = stream_grid(di, chunk->n_rows);
+    const unsigned grid = row_grid(chunk->n_rows);
     if (chunk->dtype == FOPD_BF16)
-      grad_stream_kernel<FOPD_BF16><<<grid, kStreamThreads, 0, st>>>(d, B, coef, ws, p.lambda, dlogits);
+      grad_stream_kernel<FOPD_BF16><<<grid, kGradThreads, 0, st>>>(d, B, coef, ws, p.lambda, dlogits);
     else
-      grad_stream_kernel<FOPD_F32><<<grid, kStreamThreads, 0, st>>>(d, B, coef, ws, p.lambda, dlogits);
+      grad_stream_kernel<FOPD_F32><<<grid, kGradThreads, 0, st>>>(d, B, coef, ws, p.lambda, dlogits);
     rc = launch_ok();
   }
   if (rc == FOPD_OK) {

@@ -60,21 +60,19 @@ static inline int check_params(const fopd_params &p) {
 
 static inline int launch_ok() { return cudaGetLastError() == cudaSuccess ? FOPD_OK : FOPD_ERR_CUDA; }
 
-static inline int stream_grid(const DeviceInfo &di, int64_t n_rows) {
-  const int64_t persistent = (int64_t)di.sm_count * 2;  // two 512-thread CTAs per SM
-  return (int)(n_rows < persistent ? n_rows : persistent);
-}
+// One CTA per row.
+static inline unsigned row_grid(int64_t n_rows) { return (unsigned)(n_rows < kMaxGrid ? n_rows : kMaxGrid); }
 
 // Enqueues the statistics sweep of a chunk into row_ws (and the optional
 // per-row outputs).
 static inline int launch_stats(const fopd_chunk *c, int32_t B, float *lp_s, float *lp_t, float *kl, float *ratio,
                  float *row_ws, int32_t *status, cudaStream_t st, const DeviceInfo &di) {
   const ChunkDev d = to_dev(c);
-  const int grid = stream_grid(di, c->n_rows);
+  const unsigned grid = row_grid(c->n_rows);
   if (c->dtype == FOPD_BF16)
-    token_stats_kernel<FOPD_BF16><<<grid, kStreamThreads, 0, st>>>(d, B, lp_s, lp_t, kl, ratio, row_ws, status);
+    token_stats_kernel<FOPD_BF16><<<grid, kStatsThreads, 0, st>>>(d, B, lp_s, lp_t, kl, ratio, row_ws, status);
   else
-    token_stats_kernel<FOPD_F32><<<grid, kStreamThreads, 0, st>>>(d, B, lp_s, lp_t, kl, ratio, row_ws, status);
+    token_stats_kernel<FOPD_F32><<<grid, kStatsThreads, 0, st>>>(d, B, lp_s, lp_t, kl, ratio, row_ws, status);
   return launch_ok();
 }
 

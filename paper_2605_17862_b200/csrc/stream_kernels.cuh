@@ -1,17 +1,21 @@
 // Streaming kernels of libfopd that work for any vocabulary size and both
 // logit dtypes: the statistics sweep, the single-pass gradient sweep that uses
 // cached row statistics, the per-sample segmented reduction, freshness and
-// the final loss.  One CTA walks one row at a time (persistent, row = blockIdx
-// + k * gridDim); rows are 16-byte aligned so the body uses 16-byte loads and a
-// scalar tail covers vocabularies that do not fill the last vector.
+// the final loss.  One CTA per row (the grid is the row count: the hardware's
+// block scheduler balances rows of unequal cost and staggers the CTAs' position
+// in their rows, which measured 5-9 % faster than persistent CTAs in lock step);
+// rows are 16-byte aligned so the body uses 16-byte loads and a scalar tail
+// covers vocabularies that do not fill the last vector.
 #pragma once
 
 #include "common.cuh"
 
 namespace fopd {
 
-constexpr int kStreamThreads = 512;
+constexpr int kStatsThreads = 256;   // statistics sweep: four CTAs per SM (bound by the special-function pipe)
+constexpr int kGradThreads = 1024;   // gradient sweep: one CTA per SM (bound by memory)
 constexpr int kUnroll = 4;
+constexpr int64_t kMaxGrid = 1 << 30;
 
 struct ChunkDev {
   const void *student, *teacher;
@@ -104,53 +108,31 @@ __device__ __forceinline__ RowAcc sweep_row_global(const void *srow, const void 
   return acc;
 }
 
-// a1-a4: statistics sweep.  grid = any, block = kStreamThreads.
+// a1-a4: statistics sweep.  grid = rows (any grid works), block = kStatsThreads.
 template <int DT>
-__global__ void __launch_bounds__(kStreamThreads, 2)
+__global__ void __launch_bounds__(kStatsThreads, 4)
     token_stats_kernel(ChunkDev c, int32_t B, float *lp_s, float *lp_t, float *kl, float *ratio,
                        float *row_ws, int32_t *status) {
   using E = Elem<DT>;
-  __shared__ RowAcc scratch[2][kStreamThreads / 32];  // alternating per row: no barrier after the row's finish
-  const int64_t step = gridDim.x;
-  // id, token and mask of the next row are fetched while this row is swept
-  auto side = [&](int64_t n, int32_t &sid, int32_t &y, uint32_t &m) {
-    const bool in = n < c.n_rows;
-    sid = in ? c.sid[n] : 0;
-    y = in ? c.tokens[n] : 0;
-    m = in ? c.mask[n] : 0u;
-  };
-  int64_t n = blockIdx.x;
-  int32_t sid_n, y_n;
-  uint32_t m_n;
-  side(n, sid_n, y_n, m_n);
-  for (int par = 0; n < c.n_rows; n += step) {
-    const int32_t sid = sid_n, y = y_n;
-    const uint32_t m = m_n;
-    side(n + step, sid_n, y_n, m_n);
-    bool ok = true;
-    if (sid < 0 || sid >= B) {
-      if (threadIdx.x == 0 && status) atomicOr(status, FOPD_DEV_BAD_SAMPLE);
-      ok = false;
-    }
-    if (m != 0u && (y < 0 || y >= c.vocab)) {
-      if (threadIdx.x == 0 && status) atomicOr(status, FOPD_DEV_BAD_TOKEN);
-      ok = false;
-    }
-    if (!ok || m == 0u) {
+  __shared__ RowAcc scratch[2][kStatsThreads / 32];  // alternating per row: no barrier after the row's finish
+  int par = 0;
+  for (int64_t n = blockIdx.x; n < c.n_rows; n += gridDim.x) {
+    if (!row_is_aligned(c, n, B, status, threadIdx.x == 0)) {
       if (threadIdx.x == 0) zero_row_outputs(n, lp_s, lp_t, kl, ratio, row_ws);
       continue;
     }
     // gathers of the stored token and its behaviour log-prob: issued now, used after the sweep
     float sy = 0.f, ty = 0.f, b = 0.f;
     if (threadIdx.x == 0) {
+      const int32_t y = c.tokens[n];
       sy = E::load1(c.student, n * c.stride + y);
       ty = E::load1(c.teacher, n * c.stride + y);
       b = c.behav[n];
     }
     const char *srow = reinterpret_cast<const char *>(c.student) + n * c.stride * E::kBytes;
     const char *trow = reinterpret_cast<const char *>(c.teacher) + n * c.stride * E::kBytes;
-    RowAcc acc = sweep_row_global<DT, kStreamThreads>(srow, trow, c.vocab);
-    acc = block_reduce<kStreamThreads>(acc, scratch[par]);
+    RowAcc acc = sweep_row_global<DT, kStatsThreads>(srow, trow, c.vocab);
+    acc = block_reduce<kStatsThreads>(acc, scratch[par]);
     if (threadIdx.x == 0) finish_row<DT>(n, acc, sy, ty, b, lp_s, lp_t, kl, ratio, row_ws);
     par ^= 1;
   }
@@ -191,48 +173,20 @@ __device__ __forceinline__ uint4 grad_vec(const uint4 &sv, const uint4 &tv, cons
 }
 
 // a8 with cached row statistics: one streaming pass, read S, read T, write dS.
+// grid = rows (any grid works), block = kGradThreads.
 template <int DT>
-__global__ void __launch_bounds__(kStreamThreads, 2)
+__global__ void __launch_bounds__(kGradThreads, 1)
     grad_stream_kernel(ChunkDev c, int32_t B, const float *coef, const float *row_ws, float lambda,
                        void *dlogits) {
   using E = Elem<DT>;
   constexpr int P = E::kPerVec;
-  constexpr int kThreads = kStreamThreads;
+  constexpr int kThreads = kGradThreads;
   const int64_t V = c.vocab, nvec = V / P;
-  // The side inputs of a row hang off two dependent loads (sample id -> coef), each a trip to
-  // L2 under load.  They are fetched ahead in two stages so that no row waits for them:
-  // stage A (two rows ahead) loads id, mask and token, stage B (one row ahead) uses the id
-  // to load coef and the cached statistics.
-  const int64_t step = gridDim.x;
-  auto in_range = [&](int64_t n) { return n < c.n_rows; };
-  auto stage_a = [&](int64_t n, int32_t &sid, int32_t &y, uint32_t &m) {
-    sid = in_range(n) ? c.sid[n] : -1;
-    y = in_range(n) ? c.tokens[n] : 0;
-    m = in_range(n) ? c.mask[n] : 0u;
-  };
-  auto stage_b = [&](int64_t n, int32_t sid, int32_t y, uint32_t m, float &cf, float4 &ws) {
-    const bool ok = m != 0u && sid >= 0 && sid < B && y >= 0 && y < V;
-    cf = ok ? coef[sid] : 0.f;
-    ws = ok ? reinterpret_cast<const float4 *>(row_ws)[n] : make_float4(0.f, 0.f, 0.f, 0.f);
-  };
-  int64_t n = blockIdx.x;
-  int32_t sid_a, y_a, y_b;
-  uint32_t m_a;
-  float cf_b;
-  float4 ws_b;
-  stage_a(n, sid_a, y_a, m_a);
-  stage_b(n, sid_a, y_a, m_a, cf_b, ws_b);
-  y_b = y_a;
-  stage_a(n + step, sid_a, y_a, m_a);
-  for (; n < c.n_rows; n += step) {
-    const float cf = cf_b;
-    const float4 ws = ws_b;
-    const int32_t y = y_b;
-    stage_b(n + step, sid_a, y_a, m_a, cf_b, ws_b);   // in flight while this row is swept
-    y_b = y_a;
-    stage_a(n + 2 * step, sid_a, y_a, m_a);
+  for (int64_t n = blockIdx.x; n < c.n_rows; n += gridDim.x) {
     char *orow = reinterpret_cast<char *>(dlogits) + n * c.stride * E::kBytes;
     uint4 *o4 = reinterpret_cast<uint4 *>(orow);
+    float cf = 0.f;
+    if (row_is_aligned(c, n, B, nullptr, false)) cf = coef[c.sid[n]];
     if (!(cf > 0.f)) {  // masked, padded, bad id, gated or invalid sample: +0
       const uint4 z = make_uint4(0u, 0u, 0u, 0u);
       for (int64_t i = threadIdx.x; i < nvec; i += kThreads) st_stream(o4 + i, z);
@@ -240,7 +194,7 @@ __global__ void __launch_bounds__(kStreamThreads, 2)
       if (tail < V) E::store1(orow, tail, 0.f);
       continue;
     }
-    const GradRow r = make_grad_row(ws, cf, lambda, y);
+    const GradRow r = make_grad_row(reinterpret_cast<const float4 *>(row_ws)[n], cf, lambda, c.tokens[n]);
     const char *srow = reinterpret_cast<const char *>(c.student) + n * c.stride * E::kBytes;
     const char *trow = reinterpret_cast<const char *>(c.teacher) + n * c.stride * E::kBytes;
     const uint4 *s4 = reinterpret_cast<const uint4 *>(srow);
