@@ -222,17 +222,18 @@ int fopd_loss_fwd_bwd(const fopd_chunk *chunk /* HOST */, int32_t B,
 /*
  * Launch shape fopd_loss_fwd_bwd(row_ws = NULL) uses on the current device for
  * a vocabulary and dtype: CTAs per thread-block cluster (one cluster per row),
- * slice buffers per CTA (2 = the next row's copies overlap the current row's
- * sweeps), clusters resident at once and dynamic shared memory per CTA.  All
- * outputs are HOST pointers and may be NULL.  *cluster_size = 0 means that no
- * on-chip shape fits (a row pair does not fit in sixteen CTAs' shared memory)
- * and the call runs the statistics sweep followed by the streaming gradient
- * sweep instead.  The choice is made once per (device, dtype, vocabulary) with
- * cudaOccupancyMaxActiveClusters and cached; the environment variables
- * FOPD_FUSED_CLUSTER and FOPD_FUSED_BUFS, read at that moment, pin it.
+ * threads per CTA, clusters resident at once and dynamic shared memory per CTA
+ * (three slice buffers: the copies of the row after next overlap the sweeps of
+ * the current rows).  All outputs are HOST pointers and may be NULL.
+ * *cluster_size = 0 means that no on-chip shape fits (three row pairs do not
+ * fit in sixteen CTAs' shared memory) and the call runs the statistics sweep
+ * followed by the streaming gradient sweep instead.  The choice is made once
+ * per (device, dtype, vocabulary) with cudaOccupancyMaxActiveClusters and
+ * cached; the environment variables FOPD_FUSED_CLUSTER and FOPD_FUSED_THREADS,
+ * read at that moment, pin it.
  */
 int fopd_loss_fwd_bwd_plan(int32_t dtype, int64_t vocab, int32_t *cluster_size,
-                           int32_t *slice_buffers, int32_t *resident_clusters,
+                           int32_t *block_threads, int32_t *resident_clusters,
                            int32_t *smem_bytes);
 
 /*

@@ -185,7 +185,7 @@ def fopd_loss_fwd_bwd_plan(dtype: torch.dtype, vocab: int) -> dict:
     out = [ctypes.c_int32(0) for _ in range(4)]
     _check(lib().fopd_loss_fwd_bwd_plan(FOPD_BF16 if dtype == torch.bfloat16 else FOPD_F32, int(vocab),
                                         *[ctypes.byref(o) for o in out]), "fopd_loss_fwd_bwd_plan")
-    return dict(zip(("cluster_size", "slice_buffers", "resident_clusters", "smem_bytes"),
+    return dict(zip(("cluster_size", "block_threads", "resident_clusters", "smem_bytes"),
                     (int(o.value) for o in out)))
 
 

@@ -38,9 +38,10 @@
 
 namespace fopd {
 
-constexpr int kClusterThreads = 1024;
-constexpr int kComputeWarps = kClusterThreads / 32 - 1;  // warp 0 is the control warp
-constexpr int kComputeThreads = kComputeWarps * 32;
+// Block sizes the kernel is built for.  Warp 0 is the control warp, the others compute; the
+// launcher picks the size whose compute threads share a slice most evenly (a thread sweeps
+// only a few vectors per row, so an uneven split idles a large part of the block).
+#define FOPD_CLUSTER_THREAD_CHOICES(X) X(512) X(640) X(768) X(896) X(1024)
 constexpr int kMaxClusterSize = 16;
 constexpr int kSliceBufs = 3;
 #ifndef FOPD_EXCHANGE_ASYNC
@@ -243,6 +244,8 @@ struct ClusterShared {
   float token_logit[2];                      // [row parity] S[n, y_n], written by the CTA whose slice holds it
   RowAcc warp_scratch[2][32];                // [row parity][compute warp]
   GradRow grad_row[2];                       // [row parity] constants of the gradient sweep
+  int2 token_patch[2];                       // [row parity] {compute thread that stores the token's vector or -1,
+                                             //               byte offset of the token's logit in the slice}
   int failed;
 };
 
@@ -262,7 +265,10 @@ struct FusedArgs {
 #ifdef FOPD_TRACE
 #define FOPD_TRACE_AT(id)                                                                \
   do {                                                                                   \
-    if (a.trace && blockIdx.x == 0 && tid == FOPD_TRACE_TID && k < 64) a.trace[k * 16 + (id)] = clock64(); \
+    if (a.trace && blockIdx.x == 0 && tid == FOPD_TRACE_TID && k < 64) {                 \
+      a.trace[k * 16 + (id)] = clock64();                                                \
+      a.trace[64 * 16 + k * 16 + (id)] = polls;                                          \
+    }                                                                                    \
   } while (0)
 #else
 #define FOPD_TRACE_AT(id) \
@@ -270,8 +276,8 @@ struct FusedArgs {
   } while (0)
 #endif
 
-template <int DT>
-__global__ void __launch_bounds__(kClusterThreads, 1) fused_cluster_kernel(FusedArgs a) {
+template <int DT, int kThreads>
+__global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a) {
   using E = Elem<DT>;
   constexpr int P = E::kPerVec;
   extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -287,6 +293,7 @@ __global__ void __launch_bounds__(kClusterThreads, 1) fused_cluster_kernel(Fused
   const int tid = threadIdx.x, lane = tid & 31;
   const bool control = tid < 32;
   const int ctid = tid - 32;   // index among the compute threads (negative in the control warp)
+  constexpr int n_compute = kThreads - 32, n_compute_warps = n_compute / 32;
 
   // This CTA's slice of every row, in vectors.
   const int64_t v_lo = (int64_t)rank * a.slice_vecs;
@@ -299,10 +306,10 @@ __global__ void __launch_bounds__(kClusterThreads, 1) fused_cluster_kernel(Fused
   if (tid == 0) {
     for (int b = 0; b < kSliceBufs; ++b) {
       mbar_init(smem_u32(&sh.load_bar[b]), 1);
-      mbar_init(smem_u32(&sh.free_bar[b]), kComputeWarps);
+      mbar_init(smem_u32(&sh.free_bar[b]), n_compute_warps);
     }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(smem_u32(&sh.red_bar[b]), kComputeWarps);
+      mbar_init(smem_u32(&sh.red_bar[b]), n_compute_warps);
       mbar_init(smem_u32(&sh.grad_bar[b]), 1);
       mbar_init(smem_u32(&sh.xchg_bar[b]), FOPD_EXCHANGE_ASYNC ? 1u : csize);
     }
@@ -327,9 +334,17 @@ __global__ void __launch_bounds__(kClusterThreads, 1) fused_cluster_kernel(Fused
   // After one wait has run out the rest are skipped: the results are void anyway and the
   // kernel must end soon.
   bool ok = true;
+#ifdef FOPD_TRACE
+  long long polls = 0;  // failed polls of this thread (measurement builds only)
+  auto wait_on = [&](unsigned long long *bar, uint32_t parity) {
+    while (ok && !mbar_try_wait(smem_u32(bar), parity))
+      if (++polls > (1ll << 26)) ok = false;
+  };
+#else
   auto wait_on = [&](unsigned long long *bar, uint32_t parity) {
     if (ok) ok = mbar_wait_bounded(smem_u32(bar), parity);
   };
+#endif
 
   // ---- scan over this cluster's rows, row weights fetched three rows ahead
   auto load_cf = [&](int64_t n) { return n < c.n_rows ? __ldg(a.row_cf + n) : 0.f; };
@@ -353,7 +368,7 @@ __global__ void __launch_bounds__(kClusterThreads, 1) fused_cluster_kernel(Fused
       uint4 *o4 = reinterpret_cast<uint4 *>(orow) + v_lo;
       const uint4 z = make_uint4(0u, 0u, 0u, 0u);
       if (!control)
-        for (int i = ctid; i < my_vecs; i += kComputeThreads) st_stream(o4 + i, z);
+        for (int i = ctid; i < my_vecs; i += n_compute) st_stream(o4 + i, z);
       if (has_tail) E::store1(orow, tail_idx, 0.f);
       if (rank == 0 && tid == 0) reinterpret_cast<float4 *>(a.row_ws)[n] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
@@ -388,7 +403,7 @@ __global__ void __launch_bounds__(kClusterThreads, 1) fused_cluster_kernel(Fused
         FOPD_TRACE_AT(1);
         RowAcc r;
         r.init();
-        if (lane < kComputeWarps) r = sh.warp_scratch[slot][lane];
+        if (lane < n_compute_warps) r = sh.warp_scratch[slot][lane];
         r = warp_reduce_two_step(r);
         // which CTA holds S[n, y]: the slice that contains its vector, or the last CTA for the scalar tail
         const int64_t yv = y / P;
@@ -457,6 +472,10 @@ __global__ void __launch_bounds__(kClusterThreads, 1) fused_cluster_kernel(Fused
         const float d = (sh.token_logit[slot] - ls) - b;
         if (lane == 0) {
           sh.grad_row[slot] = make_grad_row(make_float4(ls, lt, kl, d), cf_r, a.lambda, y);
+          const int64_t yl = y / P - v_lo;  // the token's vector within this CTA's slice, if it is here
+          const bool here = yl >= 0 && yl < my_vecs;
+          sh.token_patch[slot] = make_int2(here ? (int)(yl % n_compute) : -1,
+                                           here ? (int)(((int64_t)y - v_lo * P) * E::kBytes) : 0);
           mbar_arrive(smem_u32(&sh.grad_bar[slot]));
           if (rank == 0) reinterpret_cast<float4 *>(a.row_ws)[row_r] = make_float4(ls, lt, kl, d);
         }
@@ -470,7 +489,7 @@ __global__ void __launch_bounds__(kClusterThreads, 1) fused_cluster_kernel(Fused
         FOPD_TRACE_AT(1);
         SweepAcc<DT> sweep;
         sweep.init();
-        for (int i = ctid; i < my_vecs; i += kComputeThreads)
+        for (int i = ctid; i < my_vecs; i += n_compute)
           sweep.add(lds128(s_base + (uint32_t)i * 16u), lds128(t_base + (uint32_t)i * 16u));
         if (has_tail) {
           const char *srow = reinterpret_cast<const char *>(c.student) + row_r * row_bytes;
@@ -492,17 +511,16 @@ __global__ void __launch_bounds__(kClusterThreads, 1) fused_cluster_kernel(Fused
         const GradRow gr = sh.grad_row[slot ^ 1u];
         char *orow = reinterpret_cast<char *>(a.dlogits) + row_g * row_bytes;
         uint4 *o4 = reinterpret_cast<uint4 *>(orow) + v_lo;
-        for (int i = ctid; i < my_vecs; i += kComputeThreads) {
+        for (int i = ctid; i < my_vecs; i += n_compute) {
           const uint4 sv = lds128(s_base + (uint32_t)i * 16u), tv = lds128(t_base + (uint32_t)i * 16u);
           st_stream(o4 + i, grad_body<DT>(sv, tv, gr));
         }
         {
           // the stored token's element gets its extra term from the thread that wrote its vector
           // (same thread, so the two stores to that address stay in order)
-          const int64_t yv = gr.y / P - v_lo;
-          if (yv >= 0 && yv < my_vecs && (int)(yv % kComputeThreads) == ctid) {
-            const uint32_t off = (uint32_t)((int64_t)gr.y - v_lo * P) * E::kBytes;
-            const float s = lds_logit<DT>(s_base + off), t = lds_logit<DT>(t_base + off);
+          const int2 patch = sh.token_patch[slot ^ 1u];
+          if (patch.x == ctid) {
+            const float s = lds_logit<DT>(s_base + (uint32_t)patch.y), t = lds_logit<DT>(t_base + (uint32_t)patch.y);
             E::store1(orow, gr.y, fmaf(ex2(fmaf(s, kLog2e, gr.e0)), (s - t) - gr.K, gr.cg));
           }
         }

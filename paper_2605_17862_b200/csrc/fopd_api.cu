@@ -17,17 +17,25 @@ namespace {
 constexpr int kNotApplicable = 1;  // the on-chip kernel cannot take this shape; use the streaming pair
 
 // Launch shape of the on-chip kernel for one (device, dtype, vocabulary): cluster
-// size, shared memory and how many clusters are resident.
+// size, block size, shared memory and how many clusters are resident.
 struct FusedPlan {
   int cluster = 0;     // 0: no shape fits, use the streaming pair
+  int threads = 0;
   int slice_vecs = 0;
   size_t smem = 0;
   int max_clusters = 0;
 };
 
 template <int DT>
-int set_fused_attributes(int C, size_t smem) {
-  auto kernel = fused_cluster_kernel<DT>;
+const void *fused_kernel_for(int threads) {
+#define X(T) \
+  if (threads == T) return reinterpret_cast<const void *>(&fused_cluster_kernel<DT, T>);
+  FOPD_CLUSTER_THREAD_CHOICES(X)
+#undef X
+  return nullptr;
+}
+
+static int set_fused_attributes(const void *kernel, int C, size_t smem) {
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
       cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, C > 8 ? 1 : 0) != cudaSuccess) {
     (void)cudaGetLastError();
@@ -36,14 +44,14 @@ int set_fused_attributes(int C, size_t smem) {
   return FOPD_OK;
 }
 
-static void fused_launch_config(cudaLaunchConfig_t *cfg, cudaLaunchAttribute *attr, int C, size_t smem,
+static void fused_launch_config(cudaLaunchConfig_t *cfg, cudaLaunchAttribute *attr, int C, int threads, size_t smem,
                                 unsigned grid, cudaStream_t st) {
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = C;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   *cfg = cudaLaunchConfig_t{};
-  cfg->blockDim = dim3(kClusterThreads);
+  cfg->blockDim = dim3(threads);
   cfg->gridDim = dim3(grid);
   cfg->dynamicSmemBytes = smem;
   cfg->stream = st;
@@ -51,9 +59,18 @@ static void fused_launch_config(cudaLaunchConfig_t *cfg, cudaLaunchAttribute *at
   cfg->numAttrs = 1;
 }
 
-// Picks the cluster size that keeps the most CTAs resident with three slice buffers per
-// CTA (how many clusters of a given size fit depends on how the SMs are grouped), and
-// among equals the smallest.  FOPD_FUSED_CLUSTER in the environment pins the size.
+// How evenly `threads - 32` compute threads share a slice of `slice` vectors: work done
+// over work slots (1 = every thread sweeps the same number of vectors).
+static double split_efficiency(int64_t slice, int threads) {
+  const int64_t ct = threads - 32, rounds = (slice + ct - 1) / ct;
+  return rounds ? (double)slice / (double)(ct * rounds) : 0.0;
+}
+
+// Picks cluster size and block size with three slice buffers per CTA: the pair that keeps
+// the most CTAs resident (how many clusters of a given size fit depends on how the SMs are
+// grouped) weighted by how evenly the block shares its slice; among equals the smaller
+// cluster and the larger block.  FOPD_FUSED_CLUSTER / FOPD_FUSED_THREADS in the environment
+// pin them.
 template <int DT>
 int make_fused_plan(int64_t nvec, FusedPlan *plan) {
   int dev = 0, max_optin = 0;
@@ -61,28 +78,46 @@ int make_fused_plan(int64_t nvec, FusedPlan *plan) {
       cudaDeviceGetAttribute(&max_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
     return FOPD_ERR_CUDA;
   const size_t fixed = ((sizeof(ClusterShared) + 127) & ~size_t(127));
-  const char *pin_c = getenv("FOPD_FUSED_CLUSTER");
+  const char *pin_c = getenv("FOPD_FUSED_CLUSTER"), *pin_t = getenv("FOPD_FUSED_THREADS");
+  static const int choices[] = {
+#define X(T) T,
+      FOPD_CLUSTER_THREAD_CHOICES(X)
+#undef X
+  };
   FusedPlan best;
-  long best_score = 0;
+  double best_score = 0.0;
   for (int C = 1; C <= kMaxClusterSize; ++C) {
     if (pin_c && atoi(pin_c) != C) continue;
     const int64_t slice = (nvec + C - 1) / C;
     const size_t smem = fixed + (size_t)kSliceBufs * 2 * (size_t)slice * 16;
     if (smem > (size_t)max_optin || slice * 32 >= (1 << 20)) continue;  // one copy barrier counts < 2^20 bytes
-    int rc = set_fused_attributes<DT>(C, smem);
+    int threads = 0;
+    double eff = 0.0;
+    for (int t : choices) {
+      if (pin_t && atoi(pin_t) != t) continue;
+      const double e = split_efficiency(slice, t);
+      if (e >= eff) {
+        eff = e;
+        threads = t;
+      }
+    }
+    if (!threads) continue;
+    const void *kernel = fused_kernel_for<DT>(threads);
+    int rc = set_fused_attributes(kernel, C, smem);
     if (rc != FOPD_OK) return rc;
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
-    fused_launch_config(&cfg, attr, C, smem, (unsigned)C, nullptr);
+    fused_launch_config(&cfg, attr, C, threads, smem, (unsigned)C, nullptr);
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, fused_cluster_kernel<DT>, &cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) {
       (void)cudaGetLastError();
       n = 0;
     }
-    const long score = (long)n * C;
-    if (score > best_score) {
+    const double score = (double)n * C * eff;
+    if (score > best_score * 1.0001) {
       best_score = score;
       best.cluster = C;
+      best.threads = threads;
       best.slice_vecs = (int)slice;
       best.smem = smem;
       best.max_clusters = n;
@@ -127,8 +162,9 @@ int launch_fused(const fopd_chunk *chunk, int32_t B, const float *coef, float la
   if (rc != FOPD_OK) return rc;
   if (!plan.cluster || plan.max_clusters < 1) return kNotApplicable;
   const int C = plan.cluster;
+  const void *kernel = fused_kernel_for<DT>(plan.threads);
   // the attributes are per function, and the plan of another vocabulary may have changed them
-  if ((rc = set_fused_attributes<DT>(C, plan.smem)) != FOPD_OK) return rc;
+  if ((rc = set_fused_attributes(kernel, C, plan.smem)) != FOPD_OK) return rc;
   float *row_cf = tmp + 4 * chunk->n_rows;
   const ChunkDev d = to_dev(chunk);
   row_coef_kernel<<<(unsigned)((chunk->n_rows + 255) / 256), 256, 0, st>>>(d, B, coef, status, row_cf);
@@ -136,7 +172,7 @@ int launch_fused(const fopd_chunk *chunk, int32_t B, const float *coef, float la
   const int64_t clusters = chunk->n_rows < plan.max_clusters ? chunk->n_rows : plan.max_clusters;
   cudaLaunchConfig_t cfg;
   cudaLaunchAttribute attr[1];
-  fused_launch_config(&cfg, attr, C, plan.smem, (unsigned)(clusters * C), st);
+  fused_launch_config(&cfg, attr, C, plan.threads, plan.smem, (unsigned)(clusters * C), st);
   FusedArgs a;
   a.c = d;
   a.lambda = lambda;
@@ -145,7 +181,8 @@ int launch_fused(const fopd_chunk *chunk, int32_t B, const float *coef, float la
   a.row_ws = tmp;
   a.status = status;
   a.slice_vecs = plan.slice_vecs;
-  if (cudaLaunchKernelEx(&cfg, fused_cluster_kernel<DT>, a) != cudaSuccess) {
+  void *args[] = {&a};
+  if (cudaLaunchKernelExC(&cfg, kernel, args) != cudaSuccess) {
     (void)cudaGetLastError();
     return FOPD_ERR_CUDA;
   }
@@ -263,7 +300,7 @@ int fopd_loss_fwd_bwd(const fopd_chunk *chunk, int32_t B, const float *coef, con
   return rc;
 }
 
-int fopd_loss_fwd_bwd_plan(int32_t dtype, int64_t vocab, int32_t *cluster_size, int32_t *slice_buffers,
+int fopd_loss_fwd_bwd_plan(int32_t dtype, int64_t vocab, int32_t *cluster_size, int32_t *block_threads,
                            int32_t *resident_clusters, int32_t *smem_bytes) {
   if (dtype != FOPD_BF16 && dtype != FOPD_F32) return FOPD_ERR_DTYPE;
   if (vocab <= 0 || vocab > (int64_t)1 << 30) return FOPD_ERR_SIZE;
@@ -273,7 +310,7 @@ int fopd_loss_fwd_bwd_plan(int32_t dtype, int64_t vocab, int32_t *cluster_size, 
   if (nvec >= 1) rc = dtype == FOPD_BF16 ? fused_plan<FOPD_BF16>(nvec, &plan) : fused_plan<FOPD_F32>(nvec, &plan);
   if (rc != FOPD_OK) return rc;
   if (cluster_size) *cluster_size = plan.cluster;
-  if (slice_buffers) *slice_buffers = plan.cluster ? kSliceBufs : 0;
+  if (block_threads) *block_threads = plan.threads;
   if (resident_clusters) *resident_clusters = plan.max_clusters;
   if (smem_bytes) *smem_bytes = (int32_t)plan.smem;
   return FOPD_OK;
