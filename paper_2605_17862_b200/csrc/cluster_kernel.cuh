@@ -244,6 +244,7 @@ struct ClusterShared {
   float token_logit[2];                      // [row parity] S[n, y_n], written by the CTA whose slice holds it
   RowAcc warp_scratch[2][32];                // [row parity][compute warp]
   GradRow grad_row[2];                       // [row parity] constants of the gradient sweep
+  long long row_after_next[2];               // [row parity] row k + 2 of this cluster (or -1), found by the control warp
   int2 token_patch[2];                       // [row parity] {compute thread that stores the token's vector or -1,
                                              //               byte offset of the token's logit in the slice}
   int failed;
@@ -346,12 +347,24 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
   };
 #endif
 
-  // ---- scan over this cluster's rows, row weights fetched three rows ahead
+  // This CTA's part of a row that is not differentiated: zeros (compute threads only).
+  auto zero_row = [&](int64_t n) {
+    char *orow = reinterpret_cast<char *>(a.dlogits) + n * row_bytes;
+    uint4 *o4 = reinterpret_cast<uint4 *>(orow) + v_lo;
+    const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+    if (!control)
+      for (int i = ctid; i < my_vecs; i += n_compute) st_stream(o4 + i, z);
+    if (has_tail) E::store1(orow, tail_idx, 0.f);
+  };
+
+  // ---- scan over this cluster's rows, row weights fetched three rows ahead.  Every thread
+  // scans up to the first two differentiated rows; from then on only the control warp does.
   auto load_cf = [&](int64_t n) { return n < c.n_rows ? __ldg(a.row_cf + n) : 0.f; };
   int64_t scan_n = cluster_id;
   float cf0 = load_cf(scan_n), cf1 = load_cf(scan_n + n_clusters), cf2 = load_cf(scan_n + 2 * n_clusters);
-  // Next differentiated row (or -1 when the rows are exhausted); rows passed on the way are
-  // not differentiated and get their zeros here.
+  // Next differentiated row (or -1 when the rows are exhausted).  Rows passed on the way are
+  // not differentiated: they get their zeros here if compute threads take part in the call,
+  // else from the compute warps when they learn of the next row.
   auto next_row = [&](float &cf_out) -> int64_t {
     while (scan_n < c.n_rows) {
       const int64_t n = scan_n;
@@ -364,12 +377,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
         cf_out = cf;
         return n;
       }
-      char *orow = reinterpret_cast<char *>(a.dlogits) + n * row_bytes;
-      uint4 *o4 = reinterpret_cast<uint4 *>(orow) + v_lo;
-      const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-      if (!control)
-        for (int i = ctid; i < my_vecs; i += n_compute) st_stream(o4 + i, z);
-      if (has_tail) E::store1(orow, tail_idx, 0.f);
+      zero_row(n);
       if (rank == 0 && tid == 0) reinterpret_cast<float4 *>(a.row_ws)[n] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     cf_out = 0.f;
@@ -472,6 +480,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
         const float d = (sh.token_logit[slot] - ls) - b;
         if (lane == 0) {
           sh.grad_row[slot] = make_grad_row(make_float4(ls, lt, kl, d), cf_r, a.lambda, y);
+          sh.row_after_next[slot] = row_n;
           const int64_t yl = y / P - v_lo;  // the token's vector within this CTA's slice, if it is here
           const bool here = yl >= 0 && yl < my_vecs;
           sh.token_patch[slot] = make_int2(here ? (int)(yl % n_compute) : -1,
@@ -540,14 +549,28 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
         if (lane == 0) mbar_arrive(smem_u32(&sh.free_bar[buf_g]));
 #endif
       }
-      row_n = row_l >= 0 ? next_row(cf_n) : -1;
+      // The control warp scans ahead; the compute warps learn row k + 1 from the constants of
+      // row k - 1 (read above) and give the rows passed over in between their zeros.
+      if (k == 0) {
+        row_n = row_l;  // found by every thread before the loop
+      } else if (row_g >= 0) {
+        row_n = sh.row_after_next[slot ^ 1u];
+        if (row_r >= 0) {
+          const int64_t stop = row_n >= 0 ? row_n : c.n_rows;
+          for (int64_t n = row_r + n_clusters; n < stop; n += n_clusters) zero_row(n);
+        }
+      }
       FOPD_TRACE_AT(7);
     }
     row_g = row_r;
-    row_r = row_l;
-    cf_r = cf_l;
-    row_l = row_n;
-    cf_l = cf_n;
+    if (control) {
+      row_r = row_l;
+      cf_r = cf_l;
+      row_l = row_n;
+      cf_l = cf_n;
+    } else {
+      row_r = k == 0 ? row_l : row_n;  // compute warps run one row behind the control warp's scan
+    }
   }
 
   if (!ok) sh.failed = 1;
