@@ -34,7 +34,7 @@
 // the end of the kernel (the results of that call are void).
 #pragma once
 
-#include "sweep_math.cuh"
+#include "stream_kernels.cuh"
 
 namespace fopd {
 
@@ -44,12 +44,6 @@ namespace fopd {
 #define FOPD_CLUSTER_THREAD_CHOICES(X) X(512) X(640) X(768) X(896) X(1024)
 constexpr int kMaxClusterSize = 16;
 constexpr int kSliceBufs = 3;
-#ifndef FOPD_EXCHANGE_ASYNC
-#define FOPD_EXCHANGE_ASYNC 1
-#endif
-#ifndef FOPD_RELAXED_FREE
-#define FOPD_RELAXED_FREE 1
-#endif
 constexpr long long kWaitCycles = 200000000;  // SM cycles one mbarrier wait may take before giving up (~0.1 s)
 
 // ------------------------------------------------------------------ PTX wrappers
@@ -93,11 +87,6 @@ __device__ __forceinline__ void st_async_f32(uint32_t cluster_addr, float a, uin
   asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];" ::"r"(cluster_addr),
                "f"(a), "r"(cluster_bar)
                : "memory");
-}
-// Arrive on an mbarrier of another CTA of the cluster (address from mapa), releasing this
-// thread's earlier distributed-shared-memory stores to whoever acquires the barrier.
-__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -163,9 +152,6 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t local_smem, uint32_t ran
   uint32_t r;
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem), "r"(rank));
   return r;
-}
-__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
-  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
 }
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 v;
@@ -234,11 +220,7 @@ struct ClusterShared {
   unsigned long long free_bar[kSliceBufs];   // gradient sweep of the slice done (one arrival per compute warp)
   unsigned long long red_bar[2];             // [row parity] warp partials written (one arrival per compute warp)
   unsigned long long grad_bar[2];            // [row parity] grad_row ready (1 arrival)
-#if FOPD_EXCHANGE_ASYNC
   unsigned long long xchg_bar[2];            // [row parity] partials of all CTAs here (1 arrival + bytes)
-#else
-  unsigned long long xchg_bar[2];            // [row parity] partials of all CTAs here (one remote arrival per CTA)
-#endif
   float4 partial4[2][kMaxClusterSize];       // [row parity][source CTA rank] {ms, zs, as, mt}, written by peers
   float partial_zt[2][kMaxClusterSize];      // [row parity][source CTA rank] zt
   float token_logit[2];                      // [row parity] S[n, y_n], written by the CTA whose slice holds it
@@ -312,7 +294,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&sh.red_bar[b]), n_compute_warps);
       mbar_init(smem_u32(&sh.grad_bar[b]), 1);
-      mbar_init(smem_u32(&sh.xchg_bar[b]), FOPD_EXCHANGE_ASYNC ? 1u : csize);
+      mbar_init(smem_u32(&sh.xchg_bar[b]), 1);
     }
     sh.failed = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -402,10 +384,11 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
     if (control) {
       // =================================================== control warp
       int32_t y = 0;
-      float b = 0.f;
+      float b = 0.f, sy = 0.f;
       if (row_r >= 0) {
         y = c.tokens[row_r];   // used after the waits below
         b = c.behav[row_r];
+        sy = E::load1(reinterpret_cast<const char *>(c.student) + row_r * row_bytes, y);
         // CTA partial: every compute warp has written its own
         wait_on(&sh.red_bar[slot], par2);
         FOPD_TRACE_AT(1);
@@ -413,21 +396,11 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
         r.init();
         if (lane < n_compute_warps) r = sh.warp_scratch[slot][lane];
         r = warp_reduce_two_step(r);
-        // which CTA holds S[n, y]: the slice that contains its vector, or the last CTA for the scalar tail
+        // S[n, y] is sent by the CTA whose slice contains its vector (the last CTA for the scalar
+        // tail); that CTA fetched it from global memory at the top of the step
         const int64_t yv = y / P;
-        const bool in_body = yv < nvec;
-        const bool mine = in_body ? (yv >= v_lo && yv < v_lo + my_vecs) : owns_tail;
-        float sy = 0.f;
-        if (mine) {
-          if (in_body) {
-            wait_on(&sh.load_bar[buf_r], (k / kSliceBufs) & 1u);
-            sy = lds_logit<DT>(data_base + buf_r * 2u * slice_bytes + (uint32_t)((int64_t)y - v_lo * P) * E::kBytes);
-          } else {
-            sy = E::load1(reinterpret_cast<const char *>(c.student) + row_r * row_bytes, y);
-          }
-        }
+        const bool mine = yv < nvec ? (yv >= v_lo && yv < v_lo + my_vecs) : owns_tail;
         // lane j sends this CTA's partial (and the token's logit) to CTA j
-#if FOPD_EXCHANGE_ASYNC
         // every CTA (this one included) receives 20 bytes from each CTA and 4 from the token's owner
         if (lane == 0) mbar_expect_tx(smem_u32(&sh.xchg_bar[slot]), csize * 20u + 4u);
         if (lane < (int)csize) {
@@ -437,19 +410,6 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
           if (mine) st_async_f32(map_to_cta(smem_u32(&sh.token_logit[slot]), (uint32_t)lane), sy, bar);
         }
         FOPD_TRACE_AT(2);
-#else
-        if (lane < (int)csize) {
-          const uint32_t dst = map_to_cta(smem_u32(&sh.partial4[slot][rank]), (uint32_t)lane);
-          st_cluster_f32(dst + 0, r.ms);
-          st_cluster_f32(dst + 4, r.zs);
-          st_cluster_f32(dst + 8, r.as);
-          st_cluster_f32(dst + 12, r.mt);
-          st_cluster_f32(map_to_cta(smem_u32(&sh.partial_zt[slot][rank]), (uint32_t)lane), r.zt);
-          if (mine) st_cluster_f32(map_to_cta(smem_u32(&sh.token_logit[slot]), (uint32_t)lane), sy);
-          FOPD_TRACE_AT(2);
-          mbar_arrive_remote(map_to_cta(smem_u32(&sh.xchg_bar[slot]), (uint32_t)lane));
-        }
-#endif
         FOPD_TRACE_AT(3);
       }
       // look ahead: row k + 2 goes into the buffer of row k - 1 once its gradient sweep is done
@@ -496,17 +456,21 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
         const uint32_t s_base = data_base + buf_r * 2u * slice_bytes, t_base = s_base + slice_bytes;
         if (my_vecs > 0) wait_on(&sh.load_bar[buf_r], (k / kSliceBufs) & 1u);
         FOPD_TRACE_AT(1);
-        SweepAcc<DT> sweep;
+        RowAcc sweep;
         sweep.init();
-        for (int i = ctid; i < my_vecs; i += n_compute)
-          sweep.add(lds128(s_base + (uint32_t)i * 16u), lds128(t_base + (uint32_t)i * 16u));
+        for (int i = ctid; i < my_vecs; i += n_compute) {
+          float s[P], t[P];
+          E::unpack(lds128(s_base + (uint32_t)i * 16u), s);
+          E::unpack(lds128(t_base + (uint32_t)i * 16u), t);
+          sweep.add<P>(s, t);
+        }
         if (has_tail) {
           const char *srow = reinterpret_cast<const char *>(c.student) + row_r * row_bytes;
           const char *trow = reinterpret_cast<const char *>(c.teacher) + row_r * row_bytes;
           sweep.add1(E::load1(srow, tail_idx), E::load1(trow, tail_idx));
         }
         FOPD_TRACE_AT(2);
-        const RowAcc acc = warp_reduce_two_step(sweep.fold());
+        const RowAcc acc = warp_reduce_two_step(sweep);
         if (lane == 0) {
           sh.warp_scratch[slot][(tid >> 5) - 1] = acc;
           mbar_arrive(smem_u32(&sh.red_bar[slot]));
@@ -522,7 +486,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
         uint4 *o4 = reinterpret_cast<uint4 *>(orow) + v_lo;
         for (int i = ctid; i < my_vecs; i += n_compute) {
           const uint4 sv = lds128(s_base + (uint32_t)i * 16u), tv = lds128(t_base + (uint32_t)i * 16u);
-          st_stream(o4 + i, grad_body<DT>(sv, tv, gr));
+          st_stream(o4 + i, grad_vec<DT>(sv, tv, gr));
         }
         {
           // the stored token's element gets its extra term from the thread that wrote its vector
@@ -543,11 +507,7 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
         }
         FOPD_TRACE_AT(6);
         __syncwarp();
-#if FOPD_RELAXED_FREE
         if (lane == 0) mbar_arrive_relaxed(smem_u32(&sh.free_bar[buf_g]));
-#else
-        if (lane == 0) mbar_arrive(smem_u32(&sh.free_bar[buf_g]));
-#endif
       }
       // The control warp scans ahead; the compute warps learn row k + 1 from the constants of
       // row k - 1 (read above) and give the rows passed over in between their zeros.
