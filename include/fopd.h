@@ -36,9 +36,10 @@
  *
  * Memory and ownership.  Unless a parameter says HOST, every pointer is a DEVICE
  * pointer to memory the caller owns; the library keeps no pointer after a call
- * returns and has no global state.  Where a call needs temporary device memory
- * that the caller did not supply (see row_ws) it takes it from the CUDA
- * stream-ordered allocator on the caller's stream and returns it there.  All
+ * returns.  Where a call needs temporary device memory
+ * that the caller did not supply (see row_ws) it takes it from a stream-ordered
+ * memory pool of its own (one per device, which keeps the memory it has grown
+ * to) on the caller's stream and returns it there.  All
  * work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default
  * stream) and the call returns without synchronising, except
  * fopd_check_status.

@@ -222,9 +222,8 @@ int fopd_token_stats(const fopd_chunk *chunk, int32_t B, float *lp_s, float *lp_
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   float *ws = row_ws;
   if (!ws) {
-    if (cudaMallocAsync(reinterpret_cast<void **>(&ws), (size_t)chunk->n_rows * 4 * sizeof(float), st) !=
-        cudaSuccess)
-      return FOPD_ERR_CUDA;
+    if ((rc = scratch_alloc(reinterpret_cast<void **>(&ws), (size_t)chunk->n_rows * 4 * sizeof(float), st)) != FOPD_OK)
+      return rc;
   }
   rc = launch_stats(chunk, B, lp_s, lp_t, kl, ratio, ws, status, st, di);
   if (rc == FOPD_OK) {
@@ -274,9 +273,8 @@ int fopd_loss_fwd_bwd(const fopd_chunk *chunk, int32_t B, const float *coef, con
     // No cached statistics.  Preferred: the on-chip kernel, which does the reduction sweep
     // and the gradient sweep from shared memory and leaves the row statistics in tmp.
     // Shapes it cannot take fall back to the statistics sweep + streaming gradient pair.
-    if (cudaMallocAsync(reinterpret_cast<void **>(&tmp), (size_t)chunk->n_rows * 5 * sizeof(float), st) !=
-        cudaSuccess)
-      return FOPD_ERR_CUDA;
+    if ((rc = scratch_alloc(reinterpret_cast<void **>(&tmp), (size_t)chunk->n_rows * 5 * sizeof(float), st)) != FOPD_OK)
+      return rc;
     ws = tmp;
     rc = chunk->dtype == FOPD_BF16 ? launch_fused<FOPD_BF16>(chunk, B, coef, p.lambda, dlogits, tmp, status, st)
                                    : launch_fused<FOPD_F32>(chunk, B, coef, p.lambda, dlogits, tmp, status, st);

@@ -3,6 +3,7 @@
 #pragma once
 
 #include <cmath>
+#include <mutex>
 
 #include "stream_kernels.cuh"
 
@@ -59,6 +60,38 @@ static inline int check_params(const fopd_params &p) {
 }
 
 static inline int launch_ok() { return cudaGetLastError() == cudaSuccess ? FOPD_OK : FOPD_ERR_CUDA; }
+
+// Stream-ordered temporaries come from a memory pool of the library's own (one per device)
+// that keeps what it has been given: with the device's default pool a synchronisation
+// between two calls hands the memory back to the driver and the next call pays for a
+// fresh allocation, which costs more than the kernels.
+static inline int scratch_alloc(void **ptr, size_t bytes, cudaStream_t st) {
+  constexpr int kMaxDevices = 64;
+  static std::mutex mu;
+  static cudaMemPool_t pools[kMaxDevices] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return FOPD_ERR_CUDA;
+  cudaMemPool_t pool;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!pools[dev]) {
+      cudaMemPoolProps props = {};
+      props.allocType = cudaMemAllocationTypePinned;
+      props.location.type = cudaMemLocationTypeDevice;
+      props.location.id = dev;
+      cudaMemPool_t created;
+      if (cudaMemPoolCreate(&created, &props) != cudaSuccess) return FOPD_ERR_CUDA;
+      unsigned long long keep = ~0ull;
+      if (cudaMemPoolSetAttribute(created, cudaMemPoolAttrReleaseThreshold, &keep) != cudaSuccess) {
+        (void)cudaMemPoolDestroy(created);
+        return FOPD_ERR_CUDA;
+      }
+      pools[dev] = created;
+    }
+    pool = pools[dev];
+  }
+  return cudaMallocFromPoolAsync(ptr, bytes, pool, st) == cudaSuccess ? FOPD_OK : FOPD_ERR_CUDA;
+}
 
 // One CTA per row.
 static inline unsigned row_grid(int64_t n_rows) { return (unsigned)(n_rows < kMaxGrid ? n_rows : kMaxGrid); }
