@@ -182,7 +182,8 @@ int fopd_token_stats_static(const fopd_chunk *chunk /* HOST */, int32_t B, float
  *   acc        [B, 4] fp64 from fopd_token_stats (all chunks done)
  *   staleness  [B] int32 tau_i = t - r(i);  seq_len [B] int32 H_i
  *   d_sup      [B] fp32 supervision drift D_sup_i, or NULL for 0 (teacher and
- *              context unchanged since grading)
+ *              context unchanged since grading); +infinity marks a sample
+ *              without aligned supervision positions: invalid
  *   f, w, d_roll, l_distill, m_align, coef   [B] fp32 outputs; coef is
  *              required, the others may be NULL
  *   buffer_means  optional [2] fp32: mean f_i and mean m_i over the B samples
@@ -246,6 +247,61 @@ int fopd_loss_fwd_bwd_plan(int32_t dtype, int64_t vocab, int32_t *cluster_size,
 int fopd_loss_finalize(const double *loss_acc, const double *acc, const float *w,
                        int32_t B, fopd_params p, float *per_sample_loss,
                        float *loss_out, void *stream);
+
+/*
+ * Row-wise divergence diagnostics of one chunk: for every row with mask = 1 the
+ * full-vocabulary KL(p || q), p = softmax(first[n,:]), q = softmax(second[n,:]),
+ * and the entropy of p.  With first = teacher logits under the current context
+ * and second = teacher logits under the context stored at grading time, and
+ * mask = the supervision-aligned positions U^sup, the per-sample mean of the KL
+ * is the supervision drift D_sup of Eq. 10 (second row).  With first = student
+ * and second = teacher it is the token loss of Eq. 12 again, and the entropy is
+ * the response entropy the paper logs as a monitoring signal (Appendix B).
+ *
+ *   first, second   [n_rows, vocab] at a pitch of row_stride elements, same
+ *                   layout rules as fopd_chunk
+ *   mask, sample_id [n_rows]; rows with mask = 0 are not read and get 0
+ *   kl, entropy     [n_rows] fp32 outputs, either may be NULL
+ *   acc             [B, 3] fp64 {rows with mask = 1, sum kl, sum entropy} per
+ *                   sample, ADDED to in a fixed order (caller zeroes per batch)
+ */
+int fopd_row_divergence(const void *first, const void *second, const uint8_t *mask,
+                        const int32_t *sample_id, int64_t n_rows, int64_t vocab,
+                        int64_t row_stride, int32_t dtype, int32_t B, float *kl,
+                        float *entropy, double *acc, int32_t *status, void *stream);
+
+/*
+ * Per-sample supervision drift and alignment ratio from the sums of
+ * fopd_row_divergence: d_sup[i] = sum kl / |U_i^sup| (Eq. 10), m_sup[i] =
+ * |U_i^sup| / H_i (Algorithm 1), mean_entropy[i].  A sample with no aligned
+ * supervision position gets d_sup = +infinity and m_sup = 0; passed to
+ * fopd_sample_freshness that makes the sample invalid (f = w = m = coef = 0),
+ * which is Algorithm 1's |U^sup| = 0 branch.  Outputs [B] fp32, any may be NULL.
+ */
+int fopd_supervision_drift(const double *acc, const int32_t *seq_len, int32_t B,
+                           float *d_sup, float *m_sup, float *mean_entropy, void *stream);
+
+/*
+ * Buffer statistics (Eq. 14) and the adaptive-refresh rule (Eq. 15):
+ * means[0..2] = mean f_i, mean m_i^roll, mean m_i^sup over the B samples;
+ * refresh when  mean f <= kappa_f  or  mean m^roll < kappa_roll  or
+ * mean m^sup < kappa_sup  (operators as the paper prints them), but at most
+ * once every min_interval steps (Appendix B uses 200): steps_since_refresh is
+ * the number of optimizer steps since the last refresh.
+ *
+ *   f, m_roll   [B] fp32 from fopd_sample_freshness (f, m_align)
+ *   m_sup       [B] fp32 from fopd_supervision_drift, or NULL for m_roll (one
+ *               aligned set for both diagnostics)
+ *   means       [3] fp32 output or NULL
+ *   decision    [2] int32 output: decision[0] = bit 0 freshness condition, bit 1
+ *               rollout alignment, bit 2 supervision alignment, bit 3 a
+ *               condition holds but the interval has not passed;
+ *               decision[1] = 1 if the buffer is to be refreshed now
+ */
+int fopd_refresh_decision(const float *f, const float *m_roll, const float *m_sup,
+                          int32_t B, float kappa_f, float kappa_roll, float kappa_sup,
+                          int64_t steps_since_refresh, int64_t min_interval,
+                          float *means, int32_t *decision, void *stream);
 
 /* Synchronises `stream`, reads the device status word and returns FOPD_OK,
  * FOPD_ERR_DEVICE (word non-zero; *bits_out receives it if not NULL, HOST) or

@@ -18,7 +18,9 @@
  *   - the rollout drift KL(pi^t || pi^r) of Eq. 10 (first row) is estimated
  *     from the stored token y ~ pi^r alone by  k3(rho) = rho*log(rho) - rho + 1
  *     with rho = pi^t(y)/pi^r(y), whose expectation under pi^r is that KL;
- *   - both aligned sets U^roll and U^sup are the rows with mask = 1;
+ *   - the rollout-aligned set U^roll is the rows with mask = 1; the supervision
+ *     diagnostics (oracle_row_divergence) take their own mask U^sup, and the
+ *     loss path uses one set for both;
  *   - the gate w_i = ReLU(f_i - xi) is a constant in the backward pass;
  *   - the batch mean of Eq. 16 / Algorithm 1 divides by the number of samples
  *     passed in, gated and invalid ones included.
@@ -169,7 +171,9 @@ void oracle_sample_freshness(int32_t B, const double *acc, const int32_t *tau,
                              double *coef, uint8_t *valid) {
     for (int32_t i = 0; i < B; ++i) {
         double cnt = acc[3 * i];
-        int ok = cnt > 0.0 && H[i] > 0 && tau[i] >= 0;
+        /* d_sup = +inf stands for an empty supervision-aligned set: Algorithm 1
+         * marks such a sample invalid exactly like an empty rollout-aligned set. */
+        int ok = cnt > 0.0 && H[i] > 0 && tau[i] >= 0 && !(d_sup && isinf(d_sup[i]));
         valid[i] = (uint8_t)ok;
         if (!ok) {
             f[i] = w[i] = D_roll[i] = ell[i] = m[i] = coef[i] = 0.0;
@@ -185,6 +189,36 @@ void oracle_sample_freshness(int32_t B, const double *acc, const int32_t *tau,
         w[i] = g > 0.0 ? g : 0.0;
         m[i] = cnt / (double)H[i];
         coef[i] = w[i] / ((double)B * cnt);
+    }
+}
+
+/*
+ * Row-wise KL(p || q) and entropy H(p) for p = softmax(first[n,:]),
+ * q = softmax(second[n,:]) at rows with mask = 1 (zeros elsewhere).  With the
+ * teacher's logits under the current and under the stored context this is the
+ * integrand of the supervision drift D_sup, Eq. 10 second row; the entropy is
+ * the response-entropy monitoring signal of Appendix B.
+ */
+void oracle_row_divergence(const void *first, const void *second, int dtype,
+                           int64_t n_rows, int64_t V, int64_t stride,
+                           const uint8_t *mask, double *kl, double *entropy) {
+#pragma omp parallel for schedule(dynamic, 4)
+    for (int64_t n = 0; n < n_rows; ++n) {
+        kl[n] = entropy[n] = 0.0;
+        if (!mask[n]) continue;
+        size_t esz = dtype == ORACLE_BF16 ? 2 : 4;
+        const char *a = (const char *)first + (size_t)n * stride * esz;
+        const char *b = (const char *)second + (size_t)n * stride * esz;
+        double la = row_logsumexp(a, dtype, V), lb = row_logsumexp(b, dtype, V);
+        double k = 0.0, h = 0.0;
+        for (int64_t v = 0; v < V; ++v) {
+            double lp = logit_at(a, dtype, v) - la, lq = logit_at(b, dtype, v) - lb;
+            double p = exp(lp);
+            k += p * (lp - lq);
+            h -= p * lp;
+        }
+        kl[n] = k;
+        entropy[n] = h;
     }
 }
 

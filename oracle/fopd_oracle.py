@@ -187,6 +187,56 @@ def grad_rows(student, teacher, tokens, behav_logprob, mask, sample_id, coef, la
     return out
 
 
+def row_divergence(first, second, mask):
+    """Row-wise KL(softmax(first) || softmax(second)) and entropy of softmax(first)
+    at rows with mask = 1 (Eq. 10 second row when the two are the teacher under
+    the current and the stored context)."""
+    A, dt = _logits(first)
+    Bm, dt2 = _logits(second)
+    assert dt == dt2 and A.shape == Bm.shape
+    n, V = A.shape
+    mk = _np(mask, np.uint8)
+    kl, ent = np.zeros(n), np.zeros(n)
+    lib().oracle_row_divergence(_p(A), _p(Bm), ctypes.c_int(dt), ctypes.c_int64(n), ctypes.c_int64(V),
+                                ctypes.c_int64(V), _p(mk), _p(kl), _p(ent))
+    return kl, ent
+
+
+def supervision_drift(kl, entropy, mask, sample_id, H, B):
+    """D_sup_i = mean of the row KLs over U_i^sup (Eq. 10), m_sup_i = |U_i^sup| / H_i
+    (Algorithm 1), mean entropy; an empty U_i^sup gives D_sup = +inf, m_sup = 0."""
+    sid = np.asarray(sample_id)
+    m = np.asarray(mask).astype(bool)
+    H = np.asarray(H, dtype=np.float64)
+    cnt = np.zeros(B)
+    skl = np.zeros(B)
+    sen = np.zeros(B)
+    for n in range(len(sid)):  # plain loop: the definition
+        if m[n]:
+            cnt[sid[n]] += 1.0
+            skl[sid[n]] += kl[n]
+            sen[sid[n]] += entropy[n]
+    d_sup = np.where(cnt > 0, skl / np.maximum(cnt, 1.0), np.inf)
+    m_sup = np.where((cnt > 0) & (H > 0), cnt / np.where(H > 0, H, 1.0), 0.0)
+    ment = np.where(cnt > 0, sen / np.maximum(cnt, 1.0), 0.0)
+    return d_sup, m_sup, ment, cnt
+
+
+def refresh_decision(f, m_roll, m_sup, kappa_f, kappa_roll, kappa_sup, steps_since_refresh, min_interval):
+    """Eq. 14 buffer means and the Eq. 15 rule (mean f <= kappa_f or mean m < kappa),
+    at most one refresh per min_interval steps (Appendix B).  Returns (means, bits, refresh)."""
+    f = np.asarray(f, dtype=np.float64)
+    mr = np.asarray(m_roll, dtype=np.float64)
+    ms = mr if m_sup is None else np.asarray(m_sup, dtype=np.float64)
+    means = np.array([f.mean(), mr.mean(), ms.mean()])
+    bits = (1 if means[0] <= kappa_f else 0) | (2 if means[1] < kappa_roll else 0) | (4 if means[2] < kappa_sup else 0)
+    due = steps_since_refresh >= min_interval
+    refresh = bool(bits) and due
+    if bits and not due:
+        bits |= 8
+    return means, bits, refresh
+
+
 @dataclass
 class BatchResult:
     stats: list  # TokenStats per chunk

@@ -19,7 +19,8 @@ FOPD_BF16, FOPD_F32 = 0, 1
 EXPORTS = (
     "fopd_token_stats", "fopd_sample_freshness", "fopd_loss_fwd_bwd", "fopd_loss_finalize",
     "fopd_check_status", "fopd_strerror", "fopd_version", "fopd_step_host", "fopd_step_host_workspace_bytes",
-    "fopd_token_stats_static", "fopd_loss_fwd_bwd_plan",
+    "fopd_token_stats_static", "fopd_loss_fwd_bwd_plan", "fopd_row_divergence", "fopd_supervision_drift",
+    "fopd_refresh_decision",
 )
 
 
@@ -70,6 +71,10 @@ def lib() -> ctypes.CDLL:
         L.fopd_sample_freshness.argtypes = [vp, vp, vp, vp, i32, fopd_params, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.fopd_loss_fwd_bwd.argtypes = [ctypes.POINTER(fopd_chunk), i32, vp, vp, fopd_params, vp, vp, vp, vp]
         L.fopd_loss_fwd_bwd_plan.argtypes = [i32, ctypes.c_int64] + [ctypes.POINTER(ctypes.c_int32)] * 4
+        i64, f32 = ctypes.c_int64, ctypes.c_float
+        L.fopd_row_divergence.argtypes = [vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, vp, vp, vp, vp]
+        L.fopd_supervision_drift.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+        L.fopd_refresh_decision.argtypes = [vp, vp, vp, i32, f32, f32, f32, i64, i64, vp, vp, vp]
         L.fopd_loss_finalize.argtypes = [vp, vp, vp, i32, fopd_params, vp, vp, vp]
         L.fopd_check_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
         L.fopd_step_host_workspace_bytes.restype = ctypes.c_uint64
@@ -194,6 +199,29 @@ def fopd_loss_finalize(loss_acc, acc, w, B: int, p: fopd_params, loss_out, *, pe
     _check(lib().fopd_loss_finalize(_ptr(loss_acc), _ptr(acc), _ptr(w), B, p, _ptr(per_sample_loss),
                                     _ptr(loss_out), _stream(stream)),
            "fopd_loss_finalize")
+
+
+def fopd_row_divergence(first, second, mask, sample_id, B: int, acc, *, kl=None, entropy=None, vocab=None,
+                        status=None, stream=None):
+    assert first.dtype == second.dtype and first.shape == second.shape and first.stride() == second.stride()
+    n = first.shape[0]
+    _check(lib().fopd_row_divergence(_ptr(first), _ptr(second), _ptr(mask), _ptr(sample_id), n,
+                                     vocab or first.shape[1], first.stride(0) if n > 1 else first.shape[1],
+                                     FOPD_BF16 if first.dtype == torch.bfloat16 else FOPD_F32, B, _ptr(kl),
+                                     _ptr(entropy), _ptr(acc), _ptr(status), _stream(stream)),
+           "fopd_row_divergence")
+
+
+def fopd_supervision_drift(acc, seq_len, B: int, *, d_sup=None, m_sup=None, mean_entropy=None, stream=None):
+    _check(lib().fopd_supervision_drift(_ptr(acc), _ptr(seq_len), B, _ptr(d_sup), _ptr(m_sup), _ptr(mean_entropy),
+                                        _stream(stream)), "fopd_supervision_drift")
+
+
+def fopd_refresh_decision(f, m_roll, m_sup, B: int, kappa_f, kappa_roll, kappa_sup, steps_since_refresh: int,
+                          min_interval: int, decision, *, means=None, stream=None):
+    _check(lib().fopd_refresh_decision(_ptr(f), _ptr(m_roll), _ptr(m_sup), B, float(kappa_f), float(kappa_roll),
+                                       float(kappa_sup), int(steps_since_refresh), int(min_interval), _ptr(means),
+                                       _ptr(decision), _stream(stream)), "fopd_refresh_decision")
 
 
 def fopd_check_status(status, stream=None) -> int:

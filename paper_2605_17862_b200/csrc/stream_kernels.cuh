@@ -308,10 +308,11 @@ static __global__ void __launch_bounds__(256)
     if (t < 0 && status) atomicOr(status, FOPD_DEV_BAD_TAU);
     if ((h <= 0 || cnt > (double)h) && status) atomicOr(status, FOPD_DEV_BAD_LENGTH);
     double fi = 0.0, wi = 0.0, dr = 0.0, li = 0.0, mi = 0.0, ci = 0.0;
-    if (cnt > 0.0 && h > 0 && t >= 0) {
+    const double ds = d_sup ? (double)d_sup[i] : 0.0;
+    // d_sup = +inf marks a sample with no aligned supervision position: invalid (Algorithm 1)
+    if (cnt > 0.0 && h > 0 && t >= 0 && !isinf(ds)) {
       dr = acc[4 * (int64_t)i + FOPD_ACC_K3] / cnt;
       li = acc[4 * (int64_t)i + FOPD_ACC_KL] / cnt;
-      const double ds = d_sup ? (double)d_sup[i] : 0.0;
       const double surrogate = (double)p.alpha * sqrt(fmax(dr, 0.0)) + (double)p.beta * sqrt(fmax(ds, 0.0));
       fi = exp(-surrogate) / ((double)t + 1.0);
       wi = fmax(fi - (double)p.xi, 0.0);

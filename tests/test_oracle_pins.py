@@ -412,3 +412,81 @@ def test_vocabulary_permutation_invariance():
     a = orc.run_batch([chunk], 3, tau, H, None, 1.0, 1.0, 0.15, 0.1)
     p = orc.run_batch([pc], 3, tau, H, None, 1.0, 1.0, 0.15, 0.1)
     assert np.allclose(a.fresh.f, p.fresh.f, rtol=1e-13) and abs(a.loss - p.loss) < 1e-14
+
+
+# ---------------------------------------------------------------- supervision drift, entropy, refresh rule
+def test_row_divergence_matches_torch_float64_and_closed_forms():
+    g = torch.Generator().manual_seed(11)
+    A = (torch.randn(9, 37, generator=g) * 2).float()
+    Bm = (A + torch.randn(9, 37, generator=g)).float()
+    mask = np.array([1, 1, 0, 1, 1, 1, 0, 1, 1], np.uint8)
+    kl, ent = orc.row_divergence(A, Bm, mask)
+    la, lb = torch.log_softmax(A.double(), 1), torch.log_softmax(Bm.double(), 1)
+    ref_kl = torch.nn.functional.kl_div(lb, la, log_target=True, reduction="none").sum(1).numpy()
+    ref_ent = torch.distributions.Categorical(logits=A.double()).entropy().numpy()
+    m = mask.astype(bool)
+    assert np.allclose(kl[m], ref_kl[m], rtol=1e-12, atol=1e-14) and np.all(kl[~m] == 0)
+    assert np.allclose(ent[m], ref_ent[m], rtol=1e-12, atol=1e-14) and np.all(ent[~m] == 0)
+    assert np.all(kl[m] > 0)
+    # direction: KL(first || second), not the reverse
+    rev = torch.nn.functional.kl_div(la, lb, log_target=True, reduction="none").sum(1).numpy()
+    assert not np.allclose(kl[m], rev[m], rtol=1e-3)
+    # V = 2: Bernoulli closed forms
+    a = torch.tensor([[0.3, -1.1]]); b = torch.tensor([[-0.4, 0.9]])
+    p = 1 / (1 + math.exp(-(0.3 + 1.1))); q = 1 / (1 + math.exp(-(-0.4 - 0.9)))
+    k2, e2 = orc.row_divergence(a, b, np.ones(1, np.uint8))
+    assert abs(k2[0] - (p * math.log(p / q) + (1 - p) * math.log((1 - p) / (1 - q)))) < 1e-7
+    assert abs(e2[0] - (-(p * math.log(p) + (1 - p) * math.log(1 - p)))) < 1e-7
+    # identical rows: KL exactly 0; constant row: entropy log V (its maximum)
+    k0, e0 = orc.row_divergence(A, A, np.ones(9, np.uint8))
+    assert np.all(k0 == 0.0) and np.all(e0 <= math.log(37) + 1e-12)
+    _, eu = orc.row_divergence(torch.full((1, 50), 1.5), torch.zeros(1, 50), np.ones(1, np.uint8))
+    assert abs(eu[0] - math.log(50)) < 1e-12
+    # a row that puts nearly all mass on one token has entropy near 0
+    peaked = torch.zeros(1, 20); peaked[0, 3] = 60.0
+    _, ep = orc.row_divergence(peaked, torch.zeros(1, 20), np.ones(1, np.uint8))
+    assert 0 <= ep[0] < 1e-20
+
+
+def test_row_divergence_is_the_token_loss_of_eq12_for_student_and_teacher():
+    g = torch.Generator().manual_seed(12)
+    S = torch.randn(6, 19, generator=g); T = S + 0.5 * torch.randn(6, 19, generator=g)
+    st = orc.token_stats(S, T, np.zeros(6, np.int32), np.zeros(6, np.float32), np.ones(6, np.uint8),
+                         np.zeros(6, np.int32), 1)
+    kl, _ = orc.row_divergence(S, T, np.ones(6, np.uint8))
+    assert np.allclose(kl, st.kl, rtol=1e-12, atol=1e-15)
+
+
+def test_supervision_drift_means_and_empty_set():
+    kl = np.array([0.1, 0.3, 0.2, 0.7]); ent = np.array([1.0, 2.0, 3.0, 4.0])
+    d, m, e, cnt = orc.supervision_drift(kl, ent, [1, 0, 1, 0], [0, 0, 1, 2], [4, 2, 5], 3)
+    assert np.allclose(d[:2], [0.1, 0.2]) and np.isinf(d[2]) and d[2] > 0
+    assert np.allclose(m, [0.25, 0.5, 0.0]) and np.allclose(e, [1.0, 3.0, 0.0]) and np.array_equal(cnt, [1, 1, 0])
+    # an empty supervision-aligned set makes the sample invalid (Algorithm 1), whatever beta is
+    acc = np.array([[3.0, 0.03, 0.6]] * 3)
+    for beta in (0.0, 1.0):
+        fr = orc.sample_freshness(acc, [0, 1, 2], [4, 4, 4], d.astype(np.float32), 1.0, beta, 0.0)
+        assert fr.valid.tolist() == [1, 1, 0] and fr.f[2] == fr.w[2] == fr.m[2] == fr.coef[2] == 0.0
+        assert fr.f[0] > 0 and fr.f[1] > 0
+    # and D_sup enters Eq. 11 through beta * sqrt(D_sup)
+    fr = orc.sample_freshness(acc[:1], [0], [4], np.array([0.09], np.float32), 0.0, 2.0, 0.0)
+    assert abs(fr.f[0] - math.exp(-2.0 * math.sqrt(np.float32(0.09)))) < 1e-12
+
+
+def test_refresh_rule_operators_and_interval():
+    f = [0.5, 0.25, 0.75]          # mean 0.5 exactly
+    m = [0.5, 1.0, 0.75]           # mean 0.75 exactly
+    ms = [0.25, 0.25, 0.25]
+    means, bits, go = orc.refresh_decision(f, m, ms, 0.4, 0.7, 0.2, 500, 200)
+    assert np.allclose(means, [0.5, 0.75, 0.25]) and bits == 0 and not go
+    # mean f <= kappa_f triggers at equality; the alignment conditions are strict
+    assert orc.refresh_decision(f, m, ms, 0.5, 0.7, 0.2, 500, 200)[1:] == (1, True)
+    assert orc.refresh_decision(f, m, ms, 0.4, 0.75, 0.25, 500, 200)[1:] == (0, False)
+    assert orc.refresh_decision(f, m, ms, 0.4, 0.76, 0.2, 500, 200)[1:] == (2, True)
+    assert orc.refresh_decision(f, m, ms, 0.4, 0.7, 0.26, 500, 200)[1:] == (4, True)
+    assert orc.refresh_decision(f, m, ms, 0.6, 0.8, 0.3, 200, 200)[1:] == (7, True)
+    # at most one refresh per interval: the condition is reported but not acted on
+    assert orc.refresh_decision(f, m, ms, 0.6, 0.7, 0.2, 199, 200)[1:] == (1 | 8, False)
+    # one aligned set for both diagnostics: the supervision mean is the rollout mean
+    means, bits, go = orc.refresh_decision(f, m, None, 0.4, 0.7, 0.76, 500, 200)
+    assert means[2] == means[1] and bits == 4 and go
