@@ -215,3 +215,23 @@ def test_standalone_fwd_bwd_across_cluster_sizes(V):
     ch = synth.gen_chunk(wl, 0, DEV, row_block=8, row_stride=stride)
     out = par.compare([ch], B, wl.tau, wl.H, use_row_ws=False, vocab=V, grad_rows_per_chunk=12)
     print(V, out)
+
+
+def test_ablation_objectives_are_parameter_settings():
+    """The paper's compared objectives (Appendix B) are settings of the same path:
+    bare asynchronous OPD = no weighting, no anchor (w = 1: lag 0, alpha = beta = xi = 0,
+    lambda = 0: the loss is the batch mean of the per-sample mean token loss);
+    rollout-anchored regularisation only = the same with lambda > 0."""
+    wl = synth.tool_use(scale=1 / 32)
+    chunks = _chunks(wl)
+    zero_lag = np.zeros_like(wl.tau)
+    bare = dict(alpha=0.0, beta=0.0, xi=0.0, lam=0.0)
+    par.compare(chunks, wl.B, zero_lag, wl.H, params=bare, grad_rows_per_chunk=16)
+    buf, *_ = par.gpu_run(chunks, wl.B, zero_lag, wl.H, params=bare)
+    assert torch.all(buf.w == 1.0) and torch.all(buf.f == 1.0)
+    assert abs(float(buf.loss) - float(buf.l_distill.double().mean())) <= 1e-6 * float(buf.loss)
+    anchor = dict(bare, lam=0.5)
+    par.compare(chunks, wl.B, zero_lag, wl.H, params=anchor, grad_rows_per_chunk=16)
+    buf2, *_ = par.gpu_run(chunks, wl.B, zero_lag, wl.H, params=anchor)
+    want = float((buf2.l_distill.double() + 0.5 * buf2.d_roll.double()).mean())
+    assert abs(float(buf2.loss) - want) <= 1e-6 * want and float(buf2.loss) > float(buf.loss)
