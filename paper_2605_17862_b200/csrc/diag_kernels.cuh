@@ -135,8 +135,10 @@ static __global__ void __launch_bounds__(kSegThreads)
     divergence_reduce_kernel(const int32_t *sid, const uint8_t *mask, int64_t n_rows, const float2 *vals,
                              double *out) {
   __shared__ double sh[3][kSegThreads];
+  __shared__ int64_t range_sh[2];
   const int32_t i = blockIdx.x;
-  const int64_t lo = lower_bound_sid(sid, n_rows, i), hi = lower_bound_sid(sid, n_rows, i + 1);
+  int64_t lo, hi;
+  sample_row_range(sid, n_rows, i, range_sh, lo, hi);
   if (lo >= hi) return;
   double cnt = 0.0, skl = 0.0, sen = 0.0;
   for (int64_t n = lo + threadIdx.x; n < hi; n += kSegThreads) {

@@ -231,31 +231,42 @@ __global__ void __launch_bounds__(kGradThreads, 1)
 }
 
 // a5: deterministic segmented reduction of per-row statistics into per-sample
-// sums.  One block per sample; the block finds its (contiguous) row range by
-// binary search in the non-decreasing sample_id array, every thread sums a
+// sums.  One block per sample; the block finds its (contiguous) row range by a
+// parallel scan for the two places where the non-decreasing sample_id array
+// crosses its id (independent loads: a binary search is a chain of ~30 dependent
+// ones), every thread sums a
 // fixed strided subset in fp64 and a fixed tree combines them, so a rerun
 // reproduces the bits.  mode 0: acc[B,4] += {cnt, sum k3, sum kl, rows}.
 // mode 1: loss_acc[B,2] += {sum kl, sum k3} over rows of samples with coef > 0.
-constexpr int kSegThreads = 256;
+constexpr int kSegThreads = 1024;
 
-__device__ __forceinline__ int64_t lower_bound_sid(const int32_t *sid, int64_t n, int32_t key) {
-  int64_t lo = 0, hi = n;
-  while (lo < hi) {
-    const int64_t mid = (lo + hi) >> 1;
-    if (sid[mid] < key) lo = mid + 1;
-    else hi = mid;
+// First row with sample id >= key and first row with id >= key + 1 (n where there is none),
+// found by all threads of the block together; valid in every thread after the call.
+__device__ __forceinline__ void sample_row_range(const int32_t *sid, int64_t n, int32_t key, int64_t *range_sh,
+                                                 int64_t &lo, int64_t &hi) {
+  if (threadIdx.x == 0) range_sh[0] = range_sh[1] = n;
+  __syncthreads();
+  for (int64_t r = threadIdx.x; r < n; r += blockDim.x) {
+    const int32_t v = sid[r];
+    const bool first = r == 0;
+    const int32_t prev = first ? 0 : sid[r - 1];
+    if (v >= key && (first || prev < key)) range_sh[0] = r;
+    if (v > key && (first || prev <= key)) range_sh[1] = r;
   }
-  return lo;
+  __syncthreads();
+  lo = range_sh[0];
+  hi = range_sh[1];
 }
 
 static __global__ void __launch_bounds__(kSegThreads)
     segment_reduce_kernel(ChunkDev c, int32_t B, const float *row_ws, const float *coef, int mode,
                           double *out) {
   __shared__ double sh[3][kSegThreads];
+  __shared__ int64_t range_sh[2];
   const int32_t i = blockIdx.x;
   if (mode == 1 && !(coef[i] > 0.f)) return;
-  const int64_t lo = lower_bound_sid(c.sid, c.n_rows, i);
-  const int64_t hi = lower_bound_sid(c.sid, c.n_rows, i + 1);
+  int64_t lo, hi;
+  sample_row_range(c.sid, c.n_rows, i, range_sh, lo, hi);
   if (lo >= hi) return;
   double cnt = 0.0, sk3 = 0.0, skl = 0.0;
   for (int64_t n = lo + threadIdx.x; n < hi; n += kSegThreads) {
