@@ -284,10 +284,16 @@ int fopd_loss_fwd_bwd(const fopd_chunk *chunk, int32_t B, const float *coef, con
   }
   if (rc == FOPD_OK && !grad_done) {
     const unsigned grid = row_grid(chunk->n_rows);
-    if (chunk->dtype == FOPD_BF16)
-      grad_stream_kernel<FOPD_BF16><<<grid, kGradThreads, 0, st>>>(d, B, coef, ws, p.lambda, dlogits);
-    else
-      grad_stream_kernel<FOPD_F32><<<grid, kGradThreads, 0, st>>>(d, B, coef, ws, p.lambda, dlogits);
+    const bool short_row = chunk->vocab / (chunk->dtype == FOPD_BF16 ? 8 : 4) < kShortRowVecs;
+#define FOPD_LAUNCH_GRAD(DT, T) grad_stream_kernel<DT, T><<<grid, T, 0, st>>>(d, B, coef, ws, p.lambda, dlogits)
+    if (chunk->dtype == FOPD_BF16) {
+      if (short_row) FOPD_LAUNCH_GRAD(FOPD_BF16, kGradThreadsShortRow);
+      else FOPD_LAUNCH_GRAD(FOPD_BF16, kGradThreads);
+    } else {
+      if (short_row) FOPD_LAUNCH_GRAD(FOPD_F32, kGradThreadsShortRow);
+      else FOPD_LAUNCH_GRAD(FOPD_F32, kGradThreads);
+    }
+#undef FOPD_LAUNCH_GRAD
     rc = launch_ok();
   }
   if (rc == FOPD_OK) {

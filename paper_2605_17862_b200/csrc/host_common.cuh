@@ -102,10 +102,17 @@ static inline int launch_stats(const fopd_chunk *c, int32_t B, float *lp_s, floa
                  float *row_ws, int32_t *status, cudaStream_t st, const DeviceInfo &di) {
   const ChunkDev d = to_dev(c);
   const unsigned grid = row_grid(c->n_rows);
-  if (c->dtype == FOPD_BF16)
-    token_stats_kernel<FOPD_BF16><<<grid, kStatsThreads, 0, st>>>(d, B, lp_s, lp_t, kl, ratio, row_ws, status);
-  else
-    token_stats_kernel<FOPD_F32><<<grid, kStatsThreads, 0, st>>>(d, B, lp_s, lp_t, kl, ratio, row_ws, status);
+  const bool short_row = c->vocab / (c->dtype == FOPD_BF16 ? 8 : 4) < kShortRowVecs;
+#define FOPD_LAUNCH_STATS(DT, T) \
+  token_stats_kernel<DT, T><<<grid, T, 0, st>>>(d, B, lp_s, lp_t, kl, ratio, row_ws, status)
+  if (c->dtype == FOPD_BF16) {
+    if (short_row) FOPD_LAUNCH_STATS(FOPD_BF16, kStatsThreadsShortRow);
+    else FOPD_LAUNCH_STATS(FOPD_BF16, kStatsThreads);
+  } else {
+    if (short_row) FOPD_LAUNCH_STATS(FOPD_F32, kStatsThreadsShortRow);
+    else FOPD_LAUNCH_STATS(FOPD_F32, kStatsThreads);
+  }
+#undef FOPD_LAUNCH_STATS
   return launch_ok();
 }
 

@@ -12,8 +12,12 @@
 
 namespace fopd {
 
-constexpr int kStatsThreads = 256;   // statistics sweep: four CTAs per SM (bound by the special-function pipe)
-constexpr int kGradThreads = 1024;   // gradient sweep: one CTA per SM (bound by memory)
+// Block sizes by row length (measured): the statistics sweep, bound by the special-function
+// pipe, wants many small CTAs per SM; the gradient sweep, bound by memory, one or two large ones.
+// Short rows take the smaller block so that more CTAs overlap their start-up.
+constexpr int kStatsThreads = 256, kStatsThreadsShortRow = 128;
+constexpr int kGradThreads = 1024, kGradThreadsShortRow = 512;
+constexpr int64_t kShortRowVecs = 8192;  // rows of fewer 16-byte vectors count as short
 constexpr int kUnroll = 4;
 constexpr int64_t kMaxGrid = 1 << 30;
 
@@ -108,13 +112,13 @@ __device__ __forceinline__ RowAcc sweep_row_global(const void *srow, const void 
   return acc;
 }
 
-// a1-a4: statistics sweep.  grid = rows (any grid works), block = kStatsThreads.
-template <int DT>
-__global__ void __launch_bounds__(kStatsThreads, 4)
+// a1-a4: statistics sweep.  grid = rows (any grid works), block = kThreads.
+template <int DT, int kThreads>
+__global__ void __launch_bounds__(kThreads, 1024 / kThreads)
     token_stats_kernel(ChunkDev c, int32_t B, float *lp_s, float *lp_t, float *kl, float *ratio,
                        float *row_ws, int32_t *status) {
   using E = Elem<DT>;
-  __shared__ RowAcc scratch[2][kStatsThreads / 32];  // alternating per row: no barrier after the row's finish
+  __shared__ RowAcc scratch[2][kThreads / 32];  // alternating per row: no barrier after the row's finish
   int par = 0;
   for (int64_t n = blockIdx.x; n < c.n_rows; n += gridDim.x) {
     if (!row_is_aligned(c, n, B, status, threadIdx.x == 0)) {
@@ -131,8 +135,8 @@ __global__ void __launch_bounds__(kStatsThreads, 4)
     }
     const char *srow = reinterpret_cast<const char *>(c.student) + n * c.stride * E::kBytes;
     const char *trow = reinterpret_cast<const char *>(c.teacher) + n * c.stride * E::kBytes;
-    RowAcc acc = sweep_row_global<DT, kStatsThreads>(srow, trow, c.vocab);
-    acc = block_reduce<kStatsThreads>(acc, scratch[par]);
+    RowAcc acc = sweep_row_global<DT, kThreads>(srow, trow, c.vocab);
+    acc = block_reduce<kThreads>(acc, scratch[par]);
     if (threadIdx.x == 0) finish_row<DT>(n, acc, sy, ty, b, lp_s, lp_t, kl, ratio, row_ws);
     par ^= 1;
   }
@@ -173,14 +177,13 @@ __device__ __forceinline__ uint4 grad_vec(const uint4 &sv, const uint4 &tv, cons
 }
 
 // a8 with cached row statistics: one streaming pass, read S, read T, write dS.
-// grid = rows (any grid works), block = kGradThreads.
-template <int DT>
-__global__ void __launch_bounds__(kGradThreads, 1)
+// grid = rows (any grid works), block = kThreads.
+template <int DT, int kThreads>
+__global__ void __launch_bounds__(kThreads, 1024 / kThreads)
     grad_stream_kernel(ChunkDev c, int32_t B, const float *coef, const float *row_ws, float lambda,
                        void *dlogits) {
   using E = Elem<DT>;
   constexpr int P = E::kPerVec;
-  constexpr int kThreads = kGradThreads;
   const int64_t V = c.vocab, nvec = V / P;
   for (int64_t n = blockIdx.x; n < c.n_rows; n += gridDim.x) {
     char *orow = reinterpret_cast<char *>(dlogits) + n * c.stride * E::kBytes;
