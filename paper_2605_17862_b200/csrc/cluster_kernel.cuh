@@ -240,24 +240,8 @@ struct FusedArgs {
   float *row_ws;        // [n_rows,4] out: {lse_s, lse_t, kl, d}; zeros for rows not differentiated
   int32_t *status;
   int slice_vecs;       // 16-byte vectors of a row per CTA (the last CTAs' slices may be shorter or empty)
-#ifdef FOPD_TRACE
-  long long *trace;
-#endif
 };
 
-#ifdef FOPD_TRACE
-#define FOPD_TRACE_AT(id)                                                                \
-  do {                                                                                   \
-    if (a.trace && blockIdx.x == 0 && tid == FOPD_TRACE_TID && k < 64) {                 \
-      a.trace[k * 16 + (id)] = clock64();                                                \
-      a.trace[64 * 16 + k * 16 + (id)] = polls;                                          \
-    }                                                                                    \
-  } while (0)
-#else
-#define FOPD_TRACE_AT(id) \
-  do {                    \
-  } while (0)
-#endif
 
 template <int DT, int kThreads>
 __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a) {
@@ -317,17 +301,9 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
   // After one wait has run out the rest are skipped: the results are void anyway and the
   // kernel must end soon.
   bool ok = true;
-#ifdef FOPD_TRACE
-  long long polls = 0;  // failed polls of this thread (measurement builds only)
-  auto wait_on = [&](unsigned long long *bar, uint32_t parity) {
-    while (ok && !mbar_try_wait(smem_u32(bar), parity))
-      if (++polls > (1ll << 26)) ok = false;
-  };
-#else
   auto wait_on = [&](unsigned long long *bar, uint32_t parity) {
     if (ok) ok = mbar_wait_bounded(smem_u32(bar), parity);
   };
-#endif
 
   // This CTA's part of a row that is not differentiated: zeros (compute threads only).
   auto zero_row = [&](int64_t n) {
@@ -376,7 +352,6 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
   if (row_l >= 0 && tid == 0) issue_row(row_l, 1);
 
   for (uint32_t k = 0; row_r >= 0 || row_g >= 0; ++k) {
-    FOPD_TRACE_AT(0);
     const uint32_t slot = k & 1u, par2 = (k >> 1) & 1u;
     const uint32_t buf_r = k % kSliceBufs, buf_g = (k + kSliceBufs - 1) % kSliceBufs;
     float cf_n = 0.f;
@@ -391,7 +366,6 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
         sy = E::load1(reinterpret_cast<const char *>(c.student) + row_r * row_bytes, y);
         // CTA partial: every compute warp has written its own
         wait_on(&sh.red_bar[slot], par2);
-        FOPD_TRACE_AT(1);
         RowAcc r;
         r.init();
         if (lane < n_compute_warps) r = sh.warp_scratch[slot][lane];
@@ -409,21 +383,16 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
           st_async_f32(map_to_cta(smem_u32(&sh.partial_zt[slot][rank]), (uint32_t)lane), r.zt, bar);
           if (mine) st_async_f32(map_to_cta(smem_u32(&sh.token_logit[slot]), (uint32_t)lane), sy, bar);
         }
-        FOPD_TRACE_AT(2);
-        FOPD_TRACE_AT(3);
       }
       // look ahead: row k + 2 goes into the buffer of row k - 1 once its gradient sweep is done
       row_n = row_l >= 0 ? next_row(cf_n) : -1;
       if (row_n >= 0) {
         if (row_g >= 0) wait_on(&sh.free_bar[buf_g], ((k - 1) / kSliceBufs) & 1u);
-        FOPD_TRACE_AT(4);
         if (lane == 0) issue_row(row_n, (k + 2) % kSliceBufs);
-        FOPD_TRACE_AT(5);
       }
       // finish the exchange of row k: row constants, identical in every CTA
       if (row_r >= 0) {
         if (ok) ok = mbar_wait_cluster_bounded(smem_u32(&sh.xchg_bar[slot]), par2);
-        FOPD_TRACE_AT(6);
         RowAcc r;
         r.init();
         if (lane < (int)csize) {
@@ -448,14 +417,12 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
           mbar_arrive(smem_u32(&sh.grad_bar[slot]));
           if (rank == 0) reinterpret_cast<float4 *>(a.row_ws)[row_r] = make_float4(ls, lt, kl, d);
         }
-        FOPD_TRACE_AT(7);
       }
     } else {
       // =================================================== compute warps
       if (row_r >= 0) {
         const uint32_t s_base = data_base + buf_r * 2u * slice_bytes, t_base = s_base + slice_bytes;
         if (my_vecs > 0) wait_on(&sh.load_bar[buf_r], (k / kSliceBufs) & 1u);
-        FOPD_TRACE_AT(1);
         RowAcc sweep;
         sweep.init();
         for (int i = ctid; i < my_vecs; i += n_compute) {
@@ -469,18 +436,15 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
           const char *trow = reinterpret_cast<const char *>(c.teacher) + row_r * row_bytes;
           sweep.add1(E::load1(srow, tail_idx), E::load1(trow, tail_idx));
         }
-        FOPD_TRACE_AT(2);
         const RowAcc acc = warp_reduce_two_step(sweep);
         if (lane == 0) {
           sh.warp_scratch[slot][(tid >> 5) - 1] = acc;
           mbar_arrive(smem_u32(&sh.red_bar[slot]));
         }
-        FOPD_TRACE_AT(3);
       }
       if (row_g >= 0) {
         const uint32_t s_base = data_base + buf_g * 2u * slice_bytes, t_base = s_base + slice_bytes;
         wait_on(&sh.grad_bar[slot ^ 1u], ((k - 1) >> 1) & 1u);
-        FOPD_TRACE_AT(5);
         const GradRow gr = sh.grad_row[slot ^ 1u];
         char *orow = reinterpret_cast<char *>(a.dlogits) + row_g * row_bytes;
         uint4 *o4 = reinterpret_cast<uint4 *>(orow) + v_lo;
@@ -505,7 +469,6 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
           if (tail_idx == gr.y) o += gr.cg;
           E::store1(orow, tail_idx, o);
         }
-        FOPD_TRACE_AT(6);
         __syncwarp();
         if (lane == 0) mbar_arrive_relaxed(smem_u32(&sh.free_bar[buf_g]));
       }
@@ -520,7 +483,6 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
           for (int64_t n = row_r + n_clusters; n < stop; n += n_clusters) zero_row(n);
         }
       }
-      FOPD_TRACE_AT(7);
     }
     row_g = row_r;
     if (control) {

@@ -217,15 +217,13 @@ int fopd_token_stats(const fopd_chunk *chunk, int32_t B, float *lp_s, float *lp_
   if (!acc) return FOPD_ERR_NULL;
   if (row_ws && !aligned16(row_ws)) return FOPD_ERR_ALIGN;
   if (chunk->n_rows == 0) return FOPD_OK;
-  DeviceInfo di;
-  if ((rc = device_info(&di)) != FOPD_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   float *ws = row_ws;
   if (!ws) {
     if ((rc = scratch_alloc(reinterpret_cast<void **>(&ws), (size_t)chunk->n_rows * 4 * sizeof(float), st)) != FOPD_OK)
       return rc;
   }
-  rc = launch_stats(chunk, B, lp_s, lp_t, kl, ratio, ws, status, st, di);
+  rc = launch_stats(chunk, B, lp_s, lp_t, kl, ratio, ws, status, st);
   if (rc == FOPD_OK) {
     segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(to_dev(chunk), B, ws, nullptr, 0, acc);
     rc = launch_ok();
@@ -262,8 +260,6 @@ int fopd_loss_fwd_bwd(const fopd_chunk *chunk, int32_t B, const float *coef, con
     const uintptr_t o = (uintptr_t)dlogits, s = (uintptr_t)chunk->student, t = (uintptr_t)chunk->teacher;
     if ((o < s + bytes && s < o + bytes) || (o < t + bytes && t < o + bytes)) return FOPD_ERR_ALIAS;
   }
-  DeviceInfo di;
-  if ((rc = device_info(&di)) != FOPD_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const ChunkDev d = to_dev(chunk);
   const float *ws = row_ws;
@@ -280,7 +276,7 @@ int fopd_loss_fwd_bwd(const fopd_chunk *chunk, int32_t B, const float *coef, con
                                    : launch_fused<FOPD_F32>(chunk, B, coef, p.lambda, dlogits, tmp, status, st);
     if (rc == FOPD_OK) grad_done = true;
     else if (rc == kNotApplicable)
-      rc = launch_stats(chunk, B, nullptr, nullptr, nullptr, nullptr, tmp, status, st, di);
+      rc = launch_stats(chunk, B, nullptr, nullptr, nullptr, nullptr, tmp, status, st);
   }
   if (rc == FOPD_OK && !grad_done) {
     const unsigned grid = row_grid(chunk->n_rows);

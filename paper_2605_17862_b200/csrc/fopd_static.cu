@@ -45,15 +45,13 @@ extern "C" int fopd_token_stats_static(const fopd_chunk *chunk, int32_t B, float
   if (!acc) return FOPD_ERR_NULL;
   if (chunk->n_rows > FOPD_STATIC_MAX_ROWS) return FOPD_ERR_SIZE;
   if (chunk->n_rows == 0) return FOPD_OK;
-  DeviceInfo di;
-  if ((rc = device_info(&di)) != FOPD_OK) return rc;
   float *ws = nullptr;
   if ((rc = static_scratch(&ws)) != FOPD_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // The sweep writes all four scratch values of every row of the chunk (zeros
   // for rows that are not aligned) before the reduction reads them, so nothing
   // left over from an earlier call is ever read and nothing needs clearing.
-  rc = launch_stats(chunk, B, lp_s, lp_t, kl, ratio, ws, status, st, di);
+  rc = launch_stats(chunk, B, lp_s, lp_t, kl, ratio, ws, status, st);
   if (rc != FOPD_OK) return rc;
   segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(to_dev(chunk), B, ws, nullptr, 0, acc);
   return launch_ok();

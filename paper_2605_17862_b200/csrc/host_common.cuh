@@ -1,5 +1,5 @@
 // Host-side helpers shared by the entry points of libfopd: argument checks,
-// device query and the launch of the statistics sweep.
+// the memory pool for temporaries and the launch of the statistics sweep.
 #pragma once
 
 #include <cmath>
@@ -8,19 +8,6 @@
 #include "stream_kernels.cuh"
 
 namespace fopd {
-
-struct DeviceInfo {
-  int sm_count = 0;
-};
-
-static inline int device_info(DeviceInfo *out) {
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return FOPD_ERR_CUDA;
-  int sms = 0;
-  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return FOPD_ERR_CUDA;
-  out->sm_count = sms;
-  return FOPD_OK;
-}
 
 static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -99,7 +86,7 @@ static inline unsigned row_grid(int64_t n_rows) { return (unsigned)(n_rows < kMa
 // Enqueues the statistics sweep of a chunk into row_ws (and the optional
 // per-row outputs).
 static inline int launch_stats(const fopd_chunk *c, int32_t B, float *lp_s, float *lp_t, float *kl, float *ratio,
-                 float *row_ws, int32_t *status, cudaStream_t st, const DeviceInfo &di) {
+                 float *row_ws, int32_t *status, cudaStream_t st) {
   const ChunkDev d = to_dev(c);
   const unsigned grid = row_grid(c->n_rows);
   const bool short_row = c->vocab / (c->dtype == FOPD_BF16 ? 8 : 4) < kShortRowVecs;
