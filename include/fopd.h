@@ -93,7 +93,11 @@ typedef struct {
 /* One chunk of token rows.  student/teacher: [n_rows, vocab] row-major with a
  * pitch of row_stride elements (row_stride >= vocab), same dtype; base address
  * and pitch in bytes must be multiples of 16.  Rows with mask = 0 (padding,
- * tool output) are never read. */
+ * tool output) are never read.  Logits must be finite.  The sweeps subtract the
+ * row maximum before scaling and form log-probabilities and the KL from the
+ * maxima and the logs of the sums separately, so their accuracy (~1e-6) does
+ * not depend on how far the logits are from zero; only the stored
+ * log-normalisers themselves carry their fp32 rounding (6e-8 * |lse|). */
 typedef struct {
   const void *student;
   const void *teacher;

@@ -404,9 +404,10 @@ __global__ void __launch_bounds__(kThreads, 1) fused_cluster_kernel(FusedArgs a)
           r.zt = sh.partial_zt[slot][lane];
         }
         r = warp_reduce_two_step(r);
-        const float ls = r.ms + logf(r.zs), lt = r.mt + logf(r.zt);
-        const float kl = r.as / r.zs - (ls - lt);
-        const float d = (sh.token_logit[slot] - ls) - b;
+        const float gs = logf(r.zs), gt = logf(r.zt);
+        const float ls = r.ms + gs, lt = r.mt + gt;
+        const float kl = r.as / r.zs - ((r.ms - r.mt) + (gs - gt));
+        const float d = ((sh.token_logit[slot] - r.ms) - gs) - b;
         if (lane == 0) {
           sh.grad_row[slot] = make_grad_row(make_float4(ls, lt, kl, d), cf_r, a.lambda, y);
           sh.row_after_next[slot] = row_n;

@@ -130,13 +130,14 @@ struct RowAcc {
       zt *= ex2((mt - vt) * kLog2e);
       mt = vt;
     }
-    const float bs = -ms * kLog2e, bt = -mt * kLog2e;
+    // (x - max) * log2(e), not x * log2(e) - max * log2(e) in one fused multiply-add: the
+    // difference is (nearly) exact, so the result does not degrade with the size of the logits
 #pragma unroll
     for (int i = 0; i < N; ++i) {
-      const float es = ex2(fmaf(s[i], kLog2e, bs));
+      const float es = ex2((s[i] - ms) * kLog2e);
       zs += es;
       as = fmaf(es, s[i] - t[i], as);
-      zt += ex2(fmaf(t[i], kLog2e, bt));
+      zt += ex2((t[i] - mt) * kLog2e);
     }
   }
   __device__ __forceinline__ void add1(float s, float t) {

@@ -117,9 +117,10 @@ __global__ void __launch_bounds__(kDiagThreads, 4)
 #pragma unroll
       for (int off = 16; off > 0; off >>= 1) t.merge(shfl_xor(t, off));
       if (lane == 0) {
-        const float lp = t.r.ms + logf(t.r.zs), lq = t.r.mt + logf(t.r.zt);
-        const float kl = t.r.as / t.r.zs - (lp - lq);
-        const float ent = lp - t.ss / t.r.zs;
+        const float gp = logf(t.r.zs), gq = logf(t.r.zt);
+        const float kl = t.r.as / t.r.zs - ((t.r.ms - t.r.mt) + (gp - gq));
+        // H = lse - E[a] = log Z - E[a - m]: ss / zs = E[a], so subtract the maximum first
+        const float ent = gp - (t.ss / t.r.zs - t.r.ms);
         if (kl_out) kl_out[n] = kl;
         if (ent_out) ent_out[n] = ent;
         vals[n] = make_float2(kl, ent);

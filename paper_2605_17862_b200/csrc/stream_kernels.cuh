@@ -54,10 +54,12 @@ template <int DT>
 __device__ __forceinline__ void finish_row(int64_t n, const RowAcc &r, float sy, float ty, float b, float *lp_s,
                                            float *lp_t, float *kl_out, float *ratio, float *row_ws) {
   // log of the partition sums in full precision (logf, not the fast intrinsic)
-  const float ls = r.ms + logf(r.zs);
-  const float lt = r.mt + logf(r.zt);
-  const float kl = r.as / r.zs - (ls - lt);
-  const float lps = sy - ls, lpt = ty - lt;
+  // differences are formed from the maxima and the logs separately, so that they do not inherit
+  // the rounding of a large log-normaliser
+  const float gs = logf(r.zs), gt = logf(r.zt);
+  const float ls = r.ms + gs, lt = r.mt + gt;
+  const float kl = r.as / r.zs - ((r.ms - r.mt) + (gs - gt));
+  const float lps = (sy - r.ms) - gs, lpt = (ty - r.mt) - gt;
   const float d = lps - b;
   if (lp_s) lp_s[n] = lps;
   if (lp_t) lp_t[n] = lpt;

@@ -301,3 +301,20 @@ def test_on_chip_plan_is_reported():
         slice_bytes = -(-(V * e // 16) // plan["cluster_size"]) * 16
         assert plan["smem_bytes"] >= 6 * slice_bytes   # three buffers of a (student, teacher) slice pair
     assert fb.fopd_loss_fwd_bwd_plan(torch.bfloat16, 1_000_000)["cluster_size"] == 0  # falls back to streaming
+
+
+@pytest.mark.parametrize("offset,dtype", [(200.0, torch.bfloat16), (-300.0, torch.bfloat16), (100.0, torch.float32)])
+def test_large_logit_offsets(offset, dtype):
+    """Logits far from zero: a softmax is shift invariant, and the sweeps subtract the running
+    maximum before scaling, so the only loss is the fp32 rounding of the log-normaliser itself
+    (about 6e-8 * |lse|); results stay within the stated tolerances against the oracle on the
+    same shifted bits."""
+    wl = synth.tiny(scale=1 / 8) if dtype == torch.float32 else synth.reasoning(scale=1 / 32)
+    ch = synth.gen_chunk(wl, 0, DEV)
+    for k in ("student", "teacher"):
+        ch[k] = (ch[k].float() + offset).to(dtype)
+    lo, hi = wl.chunk_range(0)
+    sub = synth.Workload(wl.name, wl.B, wl.V, wl.dtype, hi - lo, wl.sample_id[lo:hi], wl.mask[lo:hi], wl.tau, wl.H)
+    for use_ws in (True, False):
+        out = par.compare([ch], sub.B, sub.tau, sub.H, use_row_ws=use_ws, grad_rows_per_chunk=32)
+    print(offset, out)
