@@ -1,14 +1,15 @@
 """GPU parity at the full benchmark sizes, in the launch configuration bench.py times.
 
-The fp64 CPU oracle cannot sweep tens of gigabytes of logits, so these tests
-check (a) every per-row output and the gradient on a seeded sample of rows that
-the oracle computes one by one -- always including the first and last row of
-every chunk and the rows on both sides of every sample boundary -- and (b)
-properties that hold at any size: the per-sample sums equal the fp64 sums of
-the per-row outputs (counts exactly), freshness / gate / weights equal the
-oracle's formulas applied to those sums, rows that are not differentiated are
-exactly +0, every differentiated row of the gradient sums to zero.  Chunks are
-streamed (generated, used, freed) exactly as the chunked configurations say.
+The fp64 CPU oracle runs its whole measurement phase over every row (chunk by
+chunk on host copies of the same bits; tens of seconds on the host cores), so
+every per-row output, the per-sample sums, freshness, gate, weights and the loss
+are compared against it with nothing taken from the CUDA path.  The gradient is
+compared on a seeded sample of rows that the oracle computes one by one -- always
+including the first and last row of every chunk and the rows on both sides of
+every sample boundary -- and, for all rows, through properties that hold at any
+size: rows that are not differentiated are exactly +0, every differentiated row
+sums to zero.  Chunks are streamed (generated, used, freed) exactly as the
+chunked configurations say.
 """
 import numpy as np
 import pytest
@@ -38,29 +39,52 @@ def _sub_chunk(ch, rows):
     return {k: v[idx].cpu() for k, v in ch.items()}
 
 
+_ORACLE_CACHE = {}
+
+
+def _oracle_measurement(wl):
+    """The oracle's measurement phase over EVERY row of the workload, chunk by chunk on host
+    copies of the same generated bits (cached per workload: two tests share `reasoning`)."""
+    if wl.name in _ORACLE_CACHE:
+        return _ORACLE_CACHE[wl.name]
+    rng = np.random.default_rng(wl.seed)
+    acc = np.zeros((wl.B, 3))
+    stats, picks, subs = [], [], []
+    for j in range(wl.n_chunks):
+        ch = synth.gen_chunk(wl, j, DEV)
+        host = {k: v.cpu() for k, v in ch.items()}
+        st = orc.token_stats(host["student"], host["teacher"], host["tokens"], host["behav_logprob"], host["mask"],
+                             host["sample_id"], wl.B)
+        orc.sample_accumulate(acc, host["sample_id"], st)
+        sel = _sample_rows(host["sample_id"].numpy(), host["student"].shape[0], rng)
+        stats.append(st)
+        picks.append(sel)
+        subs.append({k: v[torch.as_tensor(sel)].clone() for k, v in host.items()})
+        del ch, host
+    _ORACLE_CACHE[wl.name] = (stats, picks, subs, acc)
+    return _ORACLE_CACHE[wl.name]
+
+
 def _run_full_size(wl, use_row_ws):
     P = par.PARAMS
     p = fb.params(**P)
     B = wl.B
+    stats_o, picks, subs, acc_o = _oracle_measurement(wl)
+    fr = orc.sample_freshness(acc_o, wl.tau, wl.H, None, P["alpha"], P["beta"], P["xi"])
+    loss_o, per_o = orc.loss(fr, P["lam"])
     buf = pl.BatchBuffers(B, DEV)
     tau = torch.as_tensor(wl.tau, device=DEV)
     H = torch.as_tensor(wl.H, device=DEV)
-    rng = np.random.default_rng(wl.seed)
-    rows_out, picks, refs = [], [], []
+    rows_out = []
     worst = dict(lp=0.0, kl=0.0, ratio=0.0, f=0.0, loss=0.0, grad_abs=0.0, grad_rel=0.0, rowsum=0.0)
 
-    # ---- measurement phase, chunk by chunk
+    # ---- measurement phase, chunk by chunk: every per-row output of every row against the oracle
     for j in range(wl.n_chunks):
         ch = synth.gen_chunk(wl, j, DEV)
-        n = ch["student"].shape[0]
-        r = pl.RowOutputs.alloc(n, DEV)
+        r = pl.RowOutputs.alloc(ch["student"].shape[0], DEV)
         pl.measure([pl.to_chunk(ch)], buf, [r], keep_row_ws=True)
-        sel = _sample_rows(ch["sample_id"].cpu().numpy(), n, rng)
-        sub = _sub_chunk(ch, sel)
-        st = orc.token_stats(sub["student"], sub["teacher"], sub["tokens"], sub["behav_logprob"], sub["mask"],
-                             sub["sample_id"], B)
-        g = {k: getattr(r, k)[torch.as_tensor(sel, device=DEV)].cpu().numpy().astype(np.float64)
-             for k in ("lp_s", "lp_t", "kl", "ratio")}
+        st = stats_o[j]
+        g = {k: getattr(r, k).cpu().numpy().astype(np.float64) for k in ("lp_s", "lp_t", "kl", "ratio")}
         valid = st.valid.astype(bool)
         for k in g:
             assert np.all(g[k][~valid] == 0.0), k
@@ -70,13 +94,13 @@ def _run_full_size(wl, use_row_ws):
             worst["kl"] = max(worst["kl"], (np.abs(g["kl"] - st.kl) / np.maximum(1.0, st.kl))[valid].max())
             worst["ratio"] = max(worst["ratio"], (np.abs(g["ratio"] - st.rho)[valid] / st.rho[valid]).max())
         rows_out.append(r)
-        picks.append(sel)
-        refs.append((sub, st))
         del ch
     assert worst["lp"] <= par.TOL_LOGPROB and worst["kl"] <= 1e-4 and worst["ratio"] <= 1.1 * par.TOL_LOGPROB, worst
 
-    # ---- per-sample sums against fp64 sums of the per-row outputs (any-size property)
+    # ---- per-sample sums: counts exact against the oracle; and (a property that holds at any
+    # size) equal to the fp64 sums of the per-row outputs in any order
     acc = buf.acc.cpu().numpy()
+    assert np.array_equal(acc[:, 0], acc_o[:, 0]), "aligned-row counts differ"
     want = np.zeros((B, 3))
     for j, r in enumerate(rows_out):
         lo, hi = wl.chunk_range(j)
@@ -86,20 +110,25 @@ def _run_full_size(wl, use_row_ws):
         np.add.at(want[:, 0], sid[m], 1.0)
         np.add.at(want[:, 1], sid[m], np.exp(d) * d - np.expm1(d))
         np.add.at(want[:, 2], sid[m], ws[m, 2])
-    assert np.array_equal(acc[:, 0], want[:, 0]), "aligned-row counts differ"
-    assert np.allclose(acc[:, 1:3], want[:, 1:3], rtol=1e-9, atol=1e-12)
+    assert np.allclose(acc[:, :3], want, rtol=1e-9, atol=1e-12)
     assert np.array_equal(acc[:, 3], np.bincount(wl.sample_id, minlength=B).astype(np.float64))
 
-    # ---- freshness, gate, weights: the oracle's formulas on the same sums
+    # ---- freshness, gate, weights against the oracle's own sums
     pl.freshness(buf, tau, H, None, p)
-    fr = orc.sample_freshness(np.ascontiguousarray(acc[:, :3]), wl.tau, wl.H, None, P["alpha"], P["beta"], P["xi"])
     ok = fr.valid.astype(bool)
-    for name, ref in (("f", fr.f), ("w", fr.w), ("d_roll", fr.D_roll), ("l_distill", fr.ell), ("m_align", fr.m),
-                      ("coef", fr.coef)):
-        got = getattr(buf, name).cpu().numpy().astype(np.float64)
-        assert np.all(got[~ok] == 0.0), name
-        assert np.allclose(got[ok], ref[ok], rtol=1e-6, atol=1e-12), name
-    coef = buf.coef.cpu().numpy().astype(np.float64)
+    rel = lambda a, b: (np.abs(a - b) / np.maximum(np.abs(b), 1e-2))[ok].max() if ok.any() else 0.0
+    get = lambda name: getattr(buf, name).cpu().numpy().astype(np.float64)
+    for name in ("f", "w", "d_roll", "l_distill", "m_align", "coef"):
+        assert np.all(get(name)[~ok] == 0.0), name
+    worst["f"] = max(rel(get("f"), fr.f), rel(get("d_roll"), fr.D_roll), rel(get("l_distill"), fr.ell),
+                     rel(get("m_align"), fr.m))
+    assert worst["f"] <= par.TOL_REL, worst
+    assert (np.abs(get("w") - fr.w)[ok] <= par.TOL_REL * fr.f[ok]).all()
+    decided = np.abs(fr.f - P["xi"]) > 1e-5
+    assert decided[ok].all(), "a sample sits on the gate threshold: pick another seed"
+    assert np.array_equal(get("w") > 0, fr.w > 0)
+    assert (np.abs(get("coef") - fr.coef)[ok] <= par.TOL_REL * fr.f[ok] / (B * np.maximum(acc_o[ok, 0], 1))).all()
+    coef = fr.coef  # the oracle's weights: nothing below takes an input from the CUDA path
 
     # ---- optimisation phase, chunk by chunk (chunks regenerated from their seeds)
     for j in range(wl.n_chunks):
@@ -122,31 +151,29 @@ def _run_full_size(wl, use_row_ws):
                 l1 += blk.abs().sum(1)
             excess = (rs.abs() - par.out_ulp(dl.dtype) * l1).clamp_min(0.0).max()
             worst["rowsum"] = max(worst["rowsum"], float(excess) / float(coef.max()))
-        sel = picks[j]
-        sub, st = refs[j]
+        sel, sub, st = picks[j], subs[j], stats_o[j]
         g_ref = orc.grad_rows(sub["student"], sub["teacher"], sub["tokens"], sub["behav_logprob"], sub["mask"],
                               sub["sample_id"], coef, P["lam"], np.arange(len(sel)))
         g_gpu = dl[torch.as_tensor(sel, device=DEV)].double().cpu().numpy()
         err = np.abs(g_gpu - g_ref)
         worst["grad_abs"] = max(worst["grad_abs"], float(err.max()))
-        cf = coef[np.clip(sub["sample_id"].numpy(), 0, B - 1)] * st.valid
-        cp = cf[:, None] * np.exp(sub["student"].double().numpy() - st.lse_s[:, None])
+        cf = coef[np.clip(sub["sample_id"].numpy(), 0, B - 1)] * st.valid[sel]
+        cp = cf[:, None] * np.exp(sub["student"].double().numpy() - st.lse_s[sel, None])
         bound = (par.out_ulp(dl.dtype) + 2e-5) * np.abs(g_ref) + 2e-5 * cp + 1e-30
         ycol = np.clip(sub["tokens"].numpy(), 0, wl.V - 1)
-        bound[np.arange(len(sel)), ycol] += 1e-5 * np.abs(cf * P["lam"] * st.rho * (1 + np.abs(st.d)))
+        bound[np.arange(len(sel)), ycol] += 1e-5 * np.abs(cf * P["lam"] * st.rho[sel] * (1 + np.abs(st.d[sel])))
         worst["grad_rel"] = max(worst["grad_rel"], float((err / bound).max()))
         del ch, dl
     fb.fopd_loss_finalize(buf.loss_acc, buf.acc, buf.w, B, p, buf.loss, per_sample_loss=buf.per_sample_loss)
     assert fb.fopd_check_status(buf.status) == 0
     assert worst["grad_abs"] <= par.TOL_GRAD_ABS and worst["grad_rel"] <= 1.0 and worst["rowsum"] <= 1e-5, worst
 
-    # ---- loss: Eq. 16 from the oracle's per-sample means
-    total, per = orc.loss(fr, P["lam"])
+    # ---- loss (Eq. 16) against the oracle
     got = float(buf.loss.cpu()[0])
-    worst["loss"] = abs(got - total) / max(abs(total), 1e-2)
-    assert worst["loss"] <= par.TOL_REL, (got, total)
+    worst["loss"] = abs(got - loss_o) / max(abs(loss_o), 1e-2)
+    assert worst["loss"] <= par.TOL_REL, (got, loss_o)
     per_gpu = buf.per_sample_loss.cpu().numpy().astype(np.float64)
-    assert (np.abs(per_gpu - per) <= par.TOL_REL * np.maximum(np.abs(per), 1e-2)).all()
+    assert (np.abs(per_gpu - per_o) <= par.TOL_REL * np.maximum(np.abs(per_o), 1e-2)).all()
     return worst
 
 
