@@ -68,9 +68,10 @@ def test_supervision_drift_against_oracle(name):
     assert np.allclose(m.cpu().numpy(), m_o, rtol=1e-6) and np.allclose(e.cpu().numpy(), e_o, rtol=par.TOL_REL)
 
     # freshness with this D_sup: the sample without supervision positions is invalid (Algorithm 1)
+    # (the oracle's D_sup goes to both sides: no oracle input comes from the CUDA path)
     chunks = [synth.gen_chunk(wl, j, DEV) for j in range(wl.n_chunks)]
-    out = par.compare(chunks, B, wl.tau, wl.H, d_sup=dg.astype(np.float32), grad_rows_per_chunk=8)
-    buf, *_ = par.gpu_run(chunks, B, wl.tau, wl.H, d_sup=dg.astype(np.float32))
+    out = par.compare(chunks, B, wl.tau, wl.H, d_sup=d_o.astype(np.float32), grad_rows_per_chunk=8)
+    buf, *_ = par.gpu_run(chunks, B, wl.tau, wl.H, d_sup=d_o.astype(np.float32))
     assert float(buf.f[2]) == 0 and float(buf.w[2]) == 0 and float(buf.coef[2]) == 0 and float(buf.m_align[2]) == 0
     print(name, out)
 
