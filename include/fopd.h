@@ -320,7 +320,8 @@ int fopd_check_status(const int32_t *status, int32_t *bits_out /* HOST */, void 
  * (pinned memory copies fastest).
  *
  *   chunks      HOST array of n_chunks descriptors whose pointers are HOST
- *               pointers (same layout rules as for device chunks)
+ *               pointers (same layout rules as for device chunks).  The logits
+ *               of rows with mask = 0 are not uploaded (they are never read).
  *   staleness, seq_len, d_sup   HOST [B] (d_sup may be NULL)
  *   dlogits     HOST array of n_chunks HOST pointers; dlogits[j] receives
  *               chunk j's gradient, [n_rows_j, vocab] at the chunk's pitch
@@ -329,9 +330,17 @@ int fopd_check_status(const int32_t *status, int32_t *bits_out /* HOST */, void 
  *   workspace   DEVICE scratch owned by the caller, 256-byte aligned, at least
  *               fopd_step_host_workspace_bytes(.., resident = 0) bytes.  If it
  *               is at least the resident = 1 size, all logits stay on the device
- *               between the two phases and are uploaded once; otherwise every
- *               chunk is uploaded twice (once per phase).
+ *               and are uploaded once, in pieces of up to 256 MiB, on `stream`;
+ *               two library-owned streams take each piece's statistics as it
+ *               lands, differentiate a sample's rows as soon as its last row
+ *               has been measured (coef_i depends on sample i alone, Eq. 11)
+ *               and return finished gradient pieces while later rows are still
+ *               going up, so both directions of the host link are busy at once.
+ *               Otherwise every chunk is uploaded twice (once per phase) and
+ *               everything runs on `stream` in order.
  *
+ * Host-buffer steps of one process run one at a time (a lock around the shared
+ * streams); work queued on `stream` before the call is waited for first.
  * Synchronises `stream` before returning.  Returns FOPD_ERR_SIZE if the
  * workspace is too small, FOPD_ERR_DEVICE if the status word is non-zero (the
  * outputs are still written).
@@ -341,6 +350,7 @@ typedef struct {
   float *buffer_means;                                            /* [2] or NULL */
   float *loss;                                                    /* [1]         */
   int32_t *status_bits;                                           /* [1] or NULL */
+  int64_t *copied_bytes; /* [2] or NULL: bytes this call copied host->device, device->host */
 } fopd_host_outputs;
 
 uint64_t fopd_step_host_workspace_bytes(const fopd_chunk *chunks /* HOST */, int32_t n_chunks,

@@ -47,7 +47,7 @@ class fopd_chunk(ctypes.Structure):
 class fopd_host_outputs(ctypes.Structure):
     _fields_ = [(n, ctypes.c_void_p) for n in
                 ("f", "w", "d_roll", "l_distill", "m_align", "per_sample_loss", "buffer_means", "loss",
-                 "status_bits")]
+                 "status_bits", "copied_bytes")]
 
 
 _lib = None
@@ -253,7 +253,8 @@ def fopd_step_host(chunks, B: int, staleness, seq_len, d_sup, p: fopd_params, dl
     arr = _chunk_array(chunks)
     z = lambda n: torch.zeros(n, dtype=torch.float32)
     res = dict(f=z(B), w=z(B), d_roll=z(B), l_distill=z(B), m_align=z(B), per_sample_loss=z(B),
-               buffer_means=z(2), loss=z(1), status_bits=torch.zeros(1, dtype=torch.int32))
+               buffer_means=z(2), loss=z(1), status_bits=torch.zeros(1, dtype=torch.int32),
+               copied_bytes=torch.zeros(2, dtype=torch.int64))
     outs = fopd_host_outputs(*[res[n].data_ptr() for n, _ in fopd_host_outputs._fields_])
     dl = (ctypes.c_void_p * len(dlogits))(*[d.data_ptr() for d in dlogits])
     rc = lib().fopd_step_host(arr, len(chunks), B, _ptr(staleness), _ptr(seq_len), _ptr(d_sup), p, dl,

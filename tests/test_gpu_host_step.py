@@ -1,0 +1,153 @@
+"""GPU parity of the host-buffer entry point (fopd_step_host): the whole batch
+from host memory, against the fp64 CPU oracle, for both workspace sizes (all
+logits resident: uploads, kernels and downloads overlap sample by sample; small
+workspace: every chunk uploaded once per phase)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import fopd_oracle as orc
+from paper_2605_17862_b200 import binding as fb
+from paper_2605_17862_b200 import pipeline as pl
+from paper_2605_17862_b200 import synth
+
+import _parity as par
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _host_chunks(wl, row_stride=None):
+    return [{k: v.cpu().pin_memory() for k, v in synth.gen_chunk(wl, j, DEV, row_stride=row_stride).items()}
+            for j in range(wl.n_chunks)]
+
+
+def _run_host(host, B, tau, H, d_sup, params, resident, vocab=None):
+    hchunks = [pl.to_chunk(c, vocab) for c in host]
+    need = fb.fopd_step_host_workspace_bytes(hchunks, B, resident)
+    assert need > 0
+    if not resident:
+        assert need < fb.fopd_step_host_workspace_bytes(hchunks, B, True) or len(host) == 1
+    ws = torch.empty(need, dtype=torch.uint8, device=DEV)
+    dl = [torch.full_like(c["student"], float("nan")).pin_memory() for c in host]
+    res = fb.fopd_step_host(hchunks, B, torch.as_tensor(np.asarray(tau, np.int32)),
+                            torch.as_tensor(np.asarray(H, np.int32)),
+                            None if d_sup is None else torch.as_tensor(np.asarray(d_sup, np.float32)),
+                            fb.params(**params), dl, ws)
+    return res, dl
+
+
+def _check(host, B, tau, H, d_sup=None, params=par.PARAMS, resident=True, vocab=None, expect_bits=0):
+    res, dl = _run_host(host, B, tau, H, d_sup, params, resident, vocab)
+    assert int(res["status_bits"][0]) == expect_bits
+    V = vocab or host[0]["student"].shape[1]
+    hc = [dict(c) for c in host]
+    for c in hc:
+        c["student"] = c["student"][:, :V].contiguous()
+        c["teacher"] = c["teacher"][:, :V].contiguous()
+    ref = par.oracle_run(hc, B, tau, H, d_sup, params)
+    fr = ref.fresh
+    ok = fr.valid.astype(bool)
+    rel = lambda a, b: (np.abs(a.numpy().astype(np.float64) - b) / np.maximum(np.abs(b), 1e-2))[ok].max() if ok.any() else 0.0
+    assert rel(res["f"], fr.f) <= par.TOL_REL
+    assert rel(res["w"], fr.w) <= par.TOL_REL
+    assert rel(res["d_roll"], fr.D_roll) <= par.TOL_REL
+    assert rel(res["l_distill"], fr.ell) <= par.TOL_REL
+    assert rel(res["m_align"], fr.m) <= par.TOL_REL
+    for k in ("f", "w", "d_roll", "l_distill", "m_align", "per_sample_loss"):
+        assert np.all(res[k].numpy()[~ok] == 0.0), k
+    assert abs(float(res["loss"][0]) - ref.loss) <= par.TOL_REL * max(abs(ref.loss), 1e-2)
+    assert (np.abs(res["per_sample_loss"].numpy() - ref.per_sample_loss)
+            <= par.TOL_REL * np.maximum(np.abs(ref.per_sample_loss), 1e-2)).all()
+    means = res["buffer_means"].numpy()
+    assert abs(means[0] - fr.f.mean()) <= par.TOL_REL * max(fr.f.mean(), 1e-30) + 1e-12
+    assert abs(means[1] - fr.m.mean()) <= par.TOL_REL * max(fr.m.mean(), 1e-30) + 1e-12
+    worst, gmax = 0.0, 0.0
+    for j, c in enumerate(hc):
+        n = c["student"].shape[0]
+        if n == 0:
+            continue
+        g_ref = orc.grad_rows(c["student"], c["teacher"], c["tokens"], c["behav_logprob"], c["mask"],
+                              c["sample_id"], fr.coef, params["lam"], np.arange(n))
+        g = dl[j][:, :V].double().numpy()
+        assert np.isfinite(g).all(), "a gradient row was never written"
+        active = ref.stats[j].valid.astype(bool) & (fr.coef[np.clip(c["sample_id"].numpy(), 0, B - 1)] > 0)
+        assert np.all(g[~active] == 0.0) and not np.signbit(g[~active]).any()
+        worst = max(worst, float(np.abs(g - g_ref).max()))
+        gmax = max(gmax, float(np.abs(g_ref).max()))
+    assert worst <= max(par.TOL_GRAD_ABS, 1.01 * par.out_ulp(host[0]["student"].dtype) * gmax), (worst, gmax)
+    return res, dl
+
+
+@pytest.mark.parametrize("resident", [True, False])
+@pytest.mark.parametrize("name", ["tool_use", "coding_agent"])
+def test_host_step_matches_oracle(name, resident):
+    """Ragged samples that straddle chunk and piece boundaries, masked spans."""
+    wl = synth.WORKLOADS[name](scale=1 / 32)
+    assert wl.n_chunks > 1
+    _check(_host_chunks(wl), wl.B, wl.tau, wl.H, resident=resident)
+
+
+def test_host_step_tiny_config_and_device_path_agree():
+    wl = synth.tiny()
+    host = _host_chunks(wl)
+    res, dl = _check(host, wl.B, wl.tau, wl.H, resident=True)
+    dev_chunks = [{k: v.to(DEV) for k, v in c.items()} for c in host]
+    buf, _, dlog, bits = par.gpu_run(dev_chunks, wl.B, wl.tau, wl.H)
+    assert bits == 0
+    assert torch.allclose(res["loss"], buf.loss.cpu(), rtol=1e-6)
+    assert torch.allclose(res["f"], buf.f.cpu(), rtol=1e-6)
+    # same kernels, same row statistics; the weights may differ in the last place because the
+    # per-sample sums were accumulated piece by piece
+    assert torch.allclose(dl[0], dlog[0].cpu(), rtol=1e-5, atol=1e-12)
+
+
+@pytest.mark.parametrize("resident", [True, False])
+def test_host_step_edge_cases(resident):
+    """An empty chunk between two others, a sample with every row masked, a sample with no
+    rows at all, many short samples inside one piece, a supplied supervision drift, and a
+    row pitch wider than the vocabulary."""
+    rng = np.random.RandomState(11)
+    V, stride, B = 1000, 1008, 9
+    lengths = np.array([40, 3, 1, 25, 0, 7, 64, 2, 30])
+    n = int(lengths.sum())
+    sid = np.repeat(np.arange(B, dtype=np.int32), lengths)
+    mask = (rng.rand(n) > 0.3).astype(np.uint8)
+    mask[sid == 3] = 0
+    wl = synth.Workload("edge", B, V, torch.bfloat16, n, sid, mask, rng.randint(0, 4, B).astype(np.int32),
+                        np.maximum(lengths, 1).astype(np.int32), sigma_s=2.0, seed=3)
+    whole = {k: v.cpu() for k, v in synth.gen_chunk(wl, 0, DEV, row_stride=stride).items()}
+    cuts = [0, 50, 50, 51, n]
+    host = [{k: v[a:b].clone().pin_memory() for k, v in whole.items()} for a, b in zip(cuts[:-1], cuts[1:])]
+    d_sup = rng.rand(B).astype(np.float32) * 0.2
+    d_sup[8] = np.inf  # no aligned supervision position: invalid for optimisation
+    _check(host, B, wl.tau, wl.H, d_sup=d_sup, params=dict(par.PARAMS, xi=0.05), resident=resident, vocab=V)
+
+
+def test_host_step_bad_ids_set_status_bits():
+    wl = synth.tiny()
+    host = _host_chunks(wl)
+    host[0]["sample_id"][-1] = 99  # keeps the array non-decreasing
+    host[0]["tokens"][9] = wl.V + 3
+    hchunks = [pl.to_chunk(c) for c in host]
+    ws = torch.empty(fb.fopd_step_host_workspace_bytes(hchunks, wl.B, True), dtype=torch.uint8, device=DEV)
+    dl = [torch.empty_like(c["student"]).pin_memory() for c in host]
+    res = fb.fopd_step_host(hchunks, wl.B, torch.as_tensor(wl.tau), torch.as_tensor(wl.H), None,
+                            fb.params(**par.PARAMS), dl, ws)
+    bits = int(res["status_bits"][0])
+    assert bits == 1 | 2  # FOPD_DEV_BAD_TOKEN | FOPD_DEV_BAD_SAMPLE
+    assert float(dl[0][-1].abs().max()) == 0.0 and float(dl[0][9].abs().max()) == 0.0
+    assert np.isfinite(float(res["loss"][0]))
+
+
+def test_host_step_counts_the_bytes_it_copies():
+    wl = synth.tool_use(scale=1 / 32)
+    host = _host_chunks(wl)
+    res, _ = _run_host(host, wl.B, wl.tau, wl.H, None, par.PARAMS, True)
+    row = host[0]["student"].shape[1] * host[0]["student"].element_size()
+    rows = sum(c["mask"].numel() for c in host)
+    aligned = sum(int(c["mask"].sum()) for c in host)
+    h2d, d2h = (int(x) for x in res["copied_bytes"])
+    # logits of aligned rows (runs may take in short gaps), 13 bytes of side arrays per row, tau and H
+    assert 2 * row * aligned + 13 * rows + 8 * wl.B <= h2d <= 2 * row * rows + 13 * rows + 8 * wl.B
+    assert d2h == row * rows + 4 * (6 * wl.B + 2 + 1) + 4
