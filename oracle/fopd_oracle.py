@@ -237,6 +237,58 @@ def refresh_decision(f, m_roll, m_sup, kappa_f, kappa_roll, kappa_sup, steps_sin
     return means, bits, refresh
 
 
+def _to_f64(a):
+    """Logits (bf16 bit patterns, fp32, or a torch CPU tensor of either) as float64."""
+    x, dt = _logits(a)
+    if dt == BF16:
+        return (x.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    return x.astype(np.float64)
+
+
+def shard_partials(student_shard, teacher_shard, tokens, mask, v0):
+    """Partial sums of the columns [v0, v0 + W) of every row, for logits whose vocabulary
+    is split over several holders (Sec. 4.1's softmax normaliser and Eq. 12's sum, taken
+    over a part of the vocabulary): columns m_s = max s, Z_s = sum e^{s - m_s},
+    A_s = sum e^{s - m_s} (s - t), m_t, Z_t, then the stored token's two logits and a
+    flag when the token lies in this part (zeros otherwise).  Rows with mask = 0: zeros."""
+    S, T = _to_f64(student_shard), _to_f64(teacher_shard)
+    n, W = S.shape
+    y = _np(tokens, np.int64) - int(v0)
+    mk = _np(mask, np.uint8).astype(bool)
+    out = np.zeros((n, 8), dtype=np.float64)
+    for r in range(n):
+        if not mk[r]:
+            continue
+        ms, mt = S[r].max(), T[r].max()
+        es = np.exp(S[r] - ms)
+        out[r, :5] = ms, es.sum(), (es * (S[r] - T[r])).sum(), mt, np.exp(T[r] - mt).sum()
+        if 0 <= y[r] < W:
+            out[r, 5:] = S[r, y[r]], T[r, y[r]], 1.0
+    return out
+
+
+def merge_partials(parts):
+    """Whole-row normalisers, KL and stored-token logits from the partial sums of all parts
+    ([n_parts, n_rows, 8]): lse = log sum_k Z_k e^{m_k}, sum_v p_s(v)(s_v - t_v) =
+    sum_k A_k e^{m_k} / sum_k Z_k e^{m_k}.  Returns (lse_s, lse_t, kl, s_y, t_y, found)."""
+    P = np.asarray(parts, dtype=np.float64)
+    live = P[:, :, 1] > 0  # parts of rows with mask = 1
+    Ms = np.where(live, P[:, :, 0], -np.inf).max(0)
+    Mt = np.where(live, P[:, :, 3], -np.inf).max(0)
+    ok = live.any(0)
+    Ms, Mt = np.where(ok, Ms, 0.0), np.where(ok, Mt, 0.0)
+    ws = np.where(live, np.exp(P[:, :, 0] - Ms), 0.0)
+    wt = np.where(live, np.exp(P[:, :, 3] - Mt), 0.0)
+    Zs, As, Zt = (ws * P[:, :, 1]).sum(0), (ws * P[:, :, 2]).sum(0), (wt * P[:, :, 4]).sum(0)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        lse_s, lse_t = Ms + np.log(Zs), Mt + np.log(Zt)
+        kl = As / Zs - lse_s + lse_t
+    found = P[:, :, 7].sum(0)
+    sy, ty = (P[:, :, 5] * P[:, :, 7]).sum(0), (P[:, :, 6] * P[:, :, 7]).sum(0)
+    z = lambda a: np.where(ok, a, 0.0)
+    return z(lse_s), z(lse_t), z(kl), sy, ty, found
+
+
 @dataclass
 class BatchResult:
     stats: list  # TokenStats per chunk

@@ -490,3 +490,52 @@ def test_refresh_rule_operators_and_interval():
     # one aligned set for both diagnostics: the supervision mean is the rollout mean
     means, bits, go = orc.refresh_decision(f, m, None, 0.4, 0.7, 0.76, 500, 200)
     assert means[2] == means[1] and bits == 4 and go
+
+
+def test_shard_partials_hand_values_and_merge_identity():
+    # one row, parts {0, ln 2} and {ln 3}: Z over the whole row is 1 + 2 + 3 = 6
+    s = np.array([[0.0, math.log(2.0), math.log(3.0)]], np.float32)
+    t = np.zeros_like(s)
+    tok, mask = np.array([2], np.int32), np.array([1], np.uint8)
+    p0 = orc.shard_partials(s[:, :2], t[:, :2], tok, mask, 0)
+    p1 = orc.shard_partials(s[:, 2:], t[:, 2:], tok, mask, 2)
+    l2, l3 = float(np.float32(math.log(2.0))), float(np.float32(math.log(3.0)))
+    # part 0: max ln 2, Z = 1/2 + 1, A = e^{ln2 - ln2} ln 2, teacher max 0 and Z = 2, token elsewhere
+    assert np.allclose(p0[0], [l2, math.exp(-l2) + 1.0, l2, 0.0, 2.0, 0.0, 0.0, 0.0], atol=1e-12)
+    assert np.allclose(p1[0], [l3, 1.0, l3, 0.0, 1.0, l3, 0.0, 1.0], atol=1e-12)
+    lse_s, lse_t, kl, sy, ty, found = orc.merge_partials([p0, p1])
+    Z = 1.0 + math.exp(l2) + math.exp(l3)
+    assert abs(lse_s[0] - math.log(Z)) < 1e-12 and abs(lse_t[0] - math.log(3.0)) < 1e-12
+    # KL(p || uniform) = log 3 - H(p), p = (1, e^l2, e^l3) / Z
+    p = np.array([1.0, math.exp(l2), math.exp(l3)]) / Z
+    assert abs(kl[0] - (math.log(3.0) + (p * np.log(p)).sum())) < 1e-12
+    assert sy[0] == l3 and ty[0] == 0.0 and found[0] == 1.0
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_merged_shard_partials_equal_whole_row_statistics(dtype):
+    """Any split of the vocabulary gives the whole-row normalisers, KL and log-probs."""
+    rng = np.random.RandomState(7)
+    n, V, B = 9, 257, 3
+    S = torch.as_tensor(rng.randn(n, V) * 3).to(dtype)
+    T = (S.double() + torch.as_tensor(rng.randn(n, V))).to(dtype)
+    tok = rng.randint(0, V, n).astype(np.int32)
+    mask = np.array([1, 1, 0, 1, 1, 1, 0, 1, 1], np.uint8)
+    sid = np.repeat(np.arange(B, dtype=np.int32), 3)
+    b = (rng.randn(n) - 5).astype(np.float32)
+    whole = orc.token_stats(S, T, tok, b, mask, sid, B)
+    for cuts in ([0, V], [0, 1, V], [0, 100, 101, 256, V], [0, 64, 128, 192, V]):
+        parts = [orc.shard_partials(S[:, a:c].contiguous(), T[:, a:c].contiguous(), tok, mask, a)
+                 for a, c in zip(cuts[:-1], cuts[1:])]
+        lse_s, lse_t, kl, sy, ty, found = orc.merge_partials(parts)
+        ok = mask.astype(bool)
+        assert np.array_equal(found[ok], np.ones(ok.sum())) and np.all(found[~ok] == 0)
+        assert np.allclose(lse_s[ok], whole.lse_s[ok], rtol=0, atol=1e-12)
+        assert np.allclose(lse_t[ok], whole.lse_t[ok], rtol=0, atol=1e-12)
+        assert np.allclose(kl[ok], whole.kl[ok], rtol=0, atol=1e-11)
+        assert np.allclose((sy - lse_s)[ok], whole.lp_s[ok], rtol=0, atol=1e-12)
+        assert np.allclose((ty - lse_t)[ok], whole.lp_t[ok], rtol=0, atol=1e-12)
+        assert np.all(lse_s[~ok] == 0) and np.all(kl[~ok] == 0)
+    # a token outside every part is reported as not found
+    far = orc.shard_partials(S[:, :10].contiguous(), T[:, :10].contiguous(), np.full(n, 200, np.int32), mask, 0)
+    assert np.all(orc.merge_partials([far])[5] == 0)
