@@ -307,6 +307,67 @@ int fopd_refresh_decision(const float *f, const float *m_roll, const float *m_su
                           int64_t steps_since_refresh, int64_t min_interval,
                           float *means, int32_t *decision, void *stream);
 
+/*
+ * Vocabulary-sharded rows (a tensor-parallel LM head): each holder has the columns
+ * [vocab_offset, vocab_offset + shard->vocab) of every row, of a vocabulary of
+ * vocab_total columns.  The softmax normalisers of Sec. 4.1 and the sum of Eq. 12
+ * split over a partition of the vocabulary: with m_k = max, Z_k = sum e^{x - m_k}
+ * and A_k = sum e^{s - m_k}(s - t) over part k,
+ *   lse = log sum_k Z_k e^{m_k},   sum_v p_s(v)(s_v - t_v) = sum_k A_k e^{m_k} / sum_k Z_k e^{m_k}.
+ * Calling sequence on every holder, per chunk: fopd_shard_stats -> exchange the
+ * partial sums so that every holder has all parts (the caller's job: an all-gather
+ * of [n_rows, 8] floats per holder; the library makes no collective call) ->
+ * fopd_shard_merge -> (all chunks) fopd_sample_freshness -> per chunk
+ * fopd_shard_loss_fwd_bwd -> fopd_loss_finalize.  Every holder computes the same
+ * row statistics, sums, freshness and loss (the merge runs in a fixed order, part 0
+ * first) and the gradient of its own columns.
+ *
+ *   shard       DEVICE chunk whose student/teacher point at the shard's first
+ *               column of row 0 (row pitch = row_stride elements, base and pitch
+ *               16-byte aligned), vocab = columns in this shard; tokens are ids in
+ *               the FULL vocabulary; the other arrays as in fopd_chunk
+ *   partial     DEVICE [n_rows, 8] fp32 output (16-byte aligned), columns
+ *               FOPD_PART_*; rows with mask = 0 are not read and give zeros
+ */
+#define FOPD_PART_MAX_S 0
+#define FOPD_PART_Z_S 1
+#define FOPD_PART_A_S 2
+#define FOPD_PART_MAX_T 3
+#define FOPD_PART_Z_T 4
+#define FOPD_PART_TOKEN_S 5 /* student logit of the stored token, if it lies in this shard */
+#define FOPD_PART_TOKEN_T 6
+#define FOPD_PART_HAS_TOKEN 7 /* 1.0 if it does, else 0.0 */
+int fopd_shard_stats(const fopd_chunk *shard, int64_t vocab_offset, int64_t vocab_total,
+                     float *partial, void *stream);
+
+/*
+ * Merges the parts of every row into the outputs fopd_token_stats gives for
+ * unsharded rows, and adds the rows to the per-sample sums.
+ *
+ *   partials    DEVICE [n_parts, n_rows, 8] fp32, part k from the holder of the
+ *               k-th column range (any order of ranges; every column in exactly
+ *               one part)
+ *   rows        the chunk's per-row arrays (DEVICE) with vocab = vocab_total;
+ *               student, teacher and row_stride are ignored
+ *   lp_s .. ratio   optional [n_rows] outputs;  row_ws [n_rows, 4] REQUIRED
+ *   acc, status as for fopd_token_stats.  A row whose token is found in no part
+ *               or in several sets FOPD_DEV_BAD_TOKEN and is treated as masked.
+ */
+int fopd_shard_merge(const float *partials, int32_t n_parts, const fopd_chunk *rows, int32_t B,
+                     float *lp_s, float *lp_t, float *kl, float *ratio, float *row_ws,
+                     double *acc, int32_t *status, void *stream);
+
+/*
+ * Gradient of the shard's columns (same formula as fopd_loss_fwd_bwd, from the
+ * merged row statistics; one streaming pass).  dlogits has the shard's layout
+ * (DEVICE, 16-byte aligned, pitch row_stride) and must not overlap the logits.
+ * loss_acc may be NULL (the sums do not depend on the shard: every holder that
+ * passes it gets the same numbers).
+ */
+int fopd_shard_loss_fwd_bwd(const fopd_chunk *shard, int64_t vocab_offset, int64_t vocab_total,
+                            int32_t B, const float *coef, const float *row_ws, fopd_params p,
+                            void *dlogits, double *loss_acc, void *stream);
+
 /* Synchronises `stream`, reads the device status word and returns FOPD_OK,
  * FOPD_ERR_DEVICE (word non-zero; *bits_out receives it if not NULL, HOST) or
  * FOPD_ERR_CUDA. */

@@ -20,7 +20,7 @@ EXPORTS = (
     "fopd_token_stats", "fopd_sample_freshness", "fopd_loss_fwd_bwd", "fopd_loss_finalize",
     "fopd_check_status", "fopd_strerror", "fopd_version", "fopd_step_host", "fopd_step_host_workspace_bytes",
     "fopd_token_stats_static", "fopd_loss_fwd_bwd_plan", "fopd_row_divergence", "fopd_supervision_drift",
-    "fopd_refresh_decision",
+    "fopd_refresh_decision", "fopd_shard_stats", "fopd_shard_merge", "fopd_shard_loss_fwd_bwd",
 )
 
 
@@ -75,6 +75,10 @@ def lib() -> ctypes.CDLL:
         L.fopd_row_divergence.argtypes = [vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, vp, vp, vp, vp]
         L.fopd_supervision_drift.argtypes = [vp, vp, i32, vp, vp, vp, vp]
         L.fopd_refresh_decision.argtypes = [vp, vp, vp, i32, f32, f32, f32, i64, i64, vp, vp, vp]
+        L.fopd_shard_stats.argtypes = [ctypes.POINTER(fopd_chunk), i64, i64, vp, vp]
+        L.fopd_shard_merge.argtypes = [vp, i32, ctypes.POINTER(fopd_chunk), i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.fopd_shard_loss_fwd_bwd.argtypes = [ctypes.POINTER(fopd_chunk), i64, i64, i32, vp, vp, fopd_params, vp, vp,
+                                              vp]
         L.fopd_loss_finalize.argtypes = [vp, vp, vp, i32, fopd_params, vp, vp, vp]
         L.fopd_check_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
         L.fopd_step_host_workspace_bytes.restype = ctypes.c_uint64
@@ -222,6 +226,36 @@ def fopd_refresh_decision(f, m_roll, m_sup, B: int, kappa_f, kappa_roll, kappa_s
     _check(lib().fopd_refresh_decision(_ptr(f), _ptr(m_roll), _ptr(m_sup), B, float(kappa_f), float(kappa_roll),
                                        float(kappa_sup), int(steps_since_refresh), int(min_interval), _ptr(means),
                                        _ptr(decision), _stream(stream)), "fopd_refresh_decision")
+
+
+def fopd_shard_stats(shard: Chunk, vocab_offset: int, vocab_total: int, partial, *, stream=None):
+    """Partial sums [n_rows, 8] of the columns [vocab_offset, vocab_offset + W) held in ``shard``."""
+    c = shard.c_struct()
+    assert partial.dtype == torch.float32 and partial.is_contiguous() and partial.numel() == 8 * c.n_rows
+    _check(lib().fopd_shard_stats(ctypes.byref(c), int(vocab_offset), int(vocab_total), _ptr(partial),
+                                  _stream(stream)), "fopd_shard_stats")
+
+
+def fopd_shard_merge(partials, behav_logprob, tokens, mask, sample_id, vocab_total: int, B: int, acc, row_ws, *,
+                     lp_s=None, lp_t=None, kl=None, ratio=None, status=None, stream=None):
+    """Merge of all parts ([n_parts, n_rows, 8]) into the row statistics and the per-sample sums."""
+    n = tokens.numel()
+    assert partials.dtype == torch.float32 and partials.is_contiguous() and partials.dim() == 3
+    assert partials.shape[1] == n and partials.shape[2] == 8
+    rows = fopd_chunk(None, None, behav_logprob.data_ptr(), tokens.data_ptr(), mask.data_ptr(),
+                      sample_id.data_ptr(), n, int(vocab_total), int(vocab_total), FOPD_F32)
+    _check(lib().fopd_shard_merge(_ptr(partials), partials.shape[0], ctypes.byref(rows), B, _ptr(lp_s), _ptr(lp_t),
+                                  _ptr(kl), _ptr(ratio), _ptr(row_ws), _ptr(acc), _ptr(status), _stream(stream)),
+           "fopd_shard_merge")
+
+
+def fopd_shard_loss_fwd_bwd(shard: Chunk, vocab_offset: int, vocab_total: int, B: int, coef, row_ws,
+                            p: fopd_params, dlogits, *, loss_acc=None, stream=None):
+    c = shard.c_struct()
+    assert dlogits.dtype == shard.student.dtype and dlogits.stride() == shard.student.stride()
+    _check(lib().fopd_shard_loss_fwd_bwd(ctypes.byref(c), int(vocab_offset), int(vocab_total), B, _ptr(coef),
+                                         _ptr(row_ws), p, _ptr(dlogits), _ptr(loss_acc), _stream(stream)),
+           "fopd_shard_loss_fwd_bwd")
 
 
 def fopd_check_status(status, stream=None) -> int:

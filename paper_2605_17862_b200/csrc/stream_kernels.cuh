@@ -178,6 +178,58 @@ __device__ __forceinline__ uint4 grad_vec(const uint4 &sv, const uint4 &tv, cons
   return E::pack(o);
 }
 
+// A row that is not differentiated (masked, padded, bad id, gated or invalid sample): +0.
+template <int DT, int kThreads>
+__device__ __forceinline__ void zero_fill_row(char *orow, int64_t V) {
+  using E = Elem<DT>;
+  constexpr int P = E::kPerVec;
+  const int64_t nvec = V / P;
+  uint4 *o4 = reinterpret_cast<uint4 *>(orow);
+  const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+  for (int64_t i = threadIdx.x; i < nvec; i += kThreads) st_stream(o4 + i, z);
+  const int64_t tail = nvec * P + threadIdx.x;
+  if (tail < V) E::store1(orow, tail, 0.f);
+}
+
+// One streaming pass over a differentiated row: read S, read T, write dS.  r.y is the stored
+// token's column within this row view (any value outside [0, V) when it lies elsewhere).
+template <int DT, int kThreads>
+__device__ __forceinline__ void grad_row_sweep(const char *srow, const char *trow, char *orow, int64_t V,
+                                               const GradRow &r) {
+  using E = Elem<DT>;
+  constexpr int P = E::kPerVec;
+  const int64_t nvec = V / P;
+  const uint4 *s4 = reinterpret_cast<const uint4 *>(srow);
+  const uint4 *t4 = reinterpret_cast<const uint4 *>(trow);
+  uint4 *o4 = reinterpret_cast<uint4 *>(orow);
+  int64_t i = threadIdx.x;
+  for (; i + (kUnroll - 1) * kThreads < nvec; i += kUnroll * kThreads) {
+    uint4 a[kUnroll], b[kUnroll];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      a[u] = ld_stream(s4 + i + u * kThreads);
+      b[u] = ld_stream(t4 + i + u * kThreads);
+    }
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) st_stream(o4 + i + u * kThreads, grad_vec<DT>(a[u], b[u], r));
+  }
+  for (; i < nvec; i += kThreads) st_stream(o4 + i, grad_vec<DT>(ld_stream(s4 + i), ld_stream(t4 + i), r));
+  // the stored token's element: rewritten with its extra term by the thread that stored its
+  // vector (one thread, so the two stores to that address stay in order)
+  const int64_t yv = r.y / P;
+  if (r.y >= 0 && yv < nvec && (int)(yv % kThreads) == (int)threadIdx.x) {
+    const float s = E::load1(srow, r.y), t = E::load1(trow, r.y);
+    E::store1(orow, r.y, fmaf(ex2(fmaf(s, kLog2e, r.e0)), (s - t) - r.K, r.cg));
+  }
+  const int64_t tail = nvec * P + threadIdx.x;
+  if (tail < V) {
+    const float s = E::load1(srow, tail), t = E::load1(trow, tail);
+    float o = ex2(fmaf(s, kLog2e, r.e0)) * ((s - t) - r.K);
+    if (tail == r.y) o += r.cg;
+    E::store1(orow, tail, o);
+  }
+}
+
 // a8 with cached row statistics: one streaming pass, read S, read T, write dS.
 // grid = rows (any grid works), block = kThreads.
 template <int DT, int kThreads>
@@ -185,53 +237,18 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads)
     grad_stream_kernel(ChunkDev c, int32_t B, const float *coef, const float *row_ws, float lambda,
                        void *dlogits) {
   using E = Elem<DT>;
-  constexpr int P = E::kPerVec;
-  const int64_t V = c.vocab, nvec = V / P;
   for (int64_t n = blockIdx.x; n < c.n_rows; n += gridDim.x) {
     char *orow = reinterpret_cast<char *>(dlogits) + n * c.stride * E::kBytes;
-    uint4 *o4 = reinterpret_cast<uint4 *>(orow);
     float cf = 0.f;
     if (row_is_aligned(c, n, B, nullptr, false)) cf = coef[c.sid[n]];
-    if (!(cf > 0.f)) {  // masked, padded, bad id, gated or invalid sample: +0
-      const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-      for (int64_t i = threadIdx.x; i < nvec; i += kThreads) st_stream(o4 + i, z);
-      const int64_t tail = nvec * P + threadIdx.x;
-      if (tail < V) E::store1(orow, tail, 0.f);
+    if (!(cf > 0.f)) {
+      zero_fill_row<DT, kThreads>(orow, c.vocab);
       continue;
     }
     const GradRow r = make_grad_row(reinterpret_cast<const float4 *>(row_ws)[n], cf, lambda, c.tokens[n]);
-    const char *srow = reinterpret_cast<const char *>(c.student) + n * c.stride * E::kBytes;
-    const char *trow = reinterpret_cast<const char *>(c.teacher) + n * c.stride * E::kBytes;
-    const uint4 *s4 = reinterpret_cast<const uint4 *>(srow);
-    const uint4 *t4 = reinterpret_cast<const uint4 *>(trow);
-    int64_t i = threadIdx.x;
-    for (; i + (kUnroll - 1) * kThreads < nvec; i += kUnroll * kThreads) {
-      uint4 a[kUnroll], b[kUnroll];
-#pragma unroll
-      for (int u = 0; u < kUnroll; ++u) {
-        a[u] = ld_stream(s4 + i + u * kThreads);
-        b[u] = ld_stream(t4 + i + u * kThreads);
-      }
-#pragma unroll
-      for (int u = 0; u < kUnroll; ++u)
-        st_stream(o4 + i + u * kThreads, grad_vec<DT>(a[u], b[u], r));
-    }
-    for (; i < nvec; i += kThreads)
-      st_stream(o4 + i, grad_vec<DT>(ld_stream(s4 + i), ld_stream(t4 + i), r));
-    // the stored token's element: rewritten with its extra term by the thread that stored its
-    // vector (one thread, so the two stores to that address stay in order)
-    const int64_t yv = r.y / P;
-    if (yv < nvec && (int)(yv % kThreads) == (int)threadIdx.x) {
-      const float s = E::load1(srow, r.y), t = E::load1(trow, r.y);
-      E::store1(orow, r.y, fmaf(ex2(fmaf(s, kLog2e, r.e0)), (s - t) - r.K, r.cg));
-    }
-    const int64_t tail = nvec * P + threadIdx.x;
-    if (tail < V) {
-      const float s = E::load1(srow, tail), t = E::load1(trow, tail);
-      float o = ex2(fmaf(s, kLog2e, r.e0)) * ((s - t) - r.K);
-      if (tail == r.y) o += r.cg;
-      E::store1(orow, tail, o);
-    }
+    grad_row_sweep<DT, kThreads>(reinterpret_cast<const char *>(c.student) + n * c.stride * E::kBytes,
+                                 reinterpret_cast<const char *>(c.teacher) + n * c.stride * E::kBytes, orow, c.vocab,
+                                 r);
   }
 }
 

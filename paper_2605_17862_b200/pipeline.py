@@ -99,3 +99,43 @@ def step(chunks, dlogits, buf: BatchBuffers, tau, H, d_sup, p, rows=None, *, use
 
 def to_chunk(d: dict, vocab=None) -> fb.Chunk:
     return fb.Chunk(d["student"], d["teacher"], d["behav_logprob"], d["tokens"], d["mask"], d["sample_id"], vocab)
+
+
+# ---- vocabulary-sharded rows: every holder (rank) has a column range of every row ----
+
+def gather_parts(partial: torch.Tensor, group=None) -> torch.Tensor:
+    """Every holder's partial sums on every holder: [world, n_rows, 8], part k from rank k.
+    The only exchange of the sharded path (32 bytes per row and holder); one process: a copy."""
+    import torch.distributed as dist
+
+    world = dist.get_world_size(group) if dist.is_available() and dist.is_initialized() else 1
+    out = torch.empty((world,) + tuple(partial.shape), dtype=partial.dtype, device=partial.device)
+    if world == 1:
+        out[0].copy_(partial)
+    else:
+        dist.all_gather(list(out.unbind(0)), partial.contiguous(), group=group)
+    return out
+
+
+def step_vocab_sharded(shards, vocab_offset: int, vocab_total: int, dlogits, buf: BatchBuffers, tau, H, d_sup, p,
+                       rows, *, gather=gather_parts, stream=None):
+    """One pass of the whole path on a holder of the columns [vocab_offset, vocab_offset + W):
+    ``shards`` are this holder's chunks (logits = its columns, tokens = full-vocabulary ids),
+    ``rows`` one RowOutputs per chunk (row_ws is required), ``gather`` brings all holders'
+    partial sums together (default: all-gather over the default process group)."""
+    buf.reset()
+    for j, sh in enumerate(shards):
+        n = sh.tokens.numel()
+        part = torch.empty((n, 8), dtype=torch.float32, device=buf.device)
+        fb.fopd_shard_stats(sh, vocab_offset, vocab_total, part, stream=stream)
+        parts = gather(part)
+        r = rows[j]
+        fb.fopd_shard_merge(parts, sh.behav_logprob, sh.tokens, sh.mask, sh.sample_id, vocab_total, buf.B, buf.acc,
+                            r.row_ws, lp_s=r.lp_s, lp_t=r.lp_t, kl=r.kl, ratio=r.ratio, status=buf.status,
+                            stream=stream)
+    freshness(buf, tau, H, d_sup, p, stream=stream)
+    for j, sh in enumerate(shards):
+        fb.fopd_shard_loss_fwd_bwd(sh, vocab_offset, vocab_total, buf.B, buf.coef, rows[j].row_ws, p, dlogits[j],
+                                   loss_acc=buf.loss_acc, stream=stream)
+    fb.fopd_loss_finalize(buf.loss_acc, buf.acc, buf.w, buf.B, p, buf.loss,
+                          per_sample_loss=buf.per_sample_loss, stream=stream)

@@ -53,10 +53,63 @@ def out_ulp(dtype):
     return 2.0 ** -8 if dtype == torch.bfloat16 else 2.0 ** -24
 
 
+def gpu_run_vocab_sharded(cuts):
+    """A runner with gpu_run's signature that splits the vocabulary at ``cuts`` (column
+    indices, first 0, last V) and plays every holder in turn on the one GPU: all holders'
+    partial sums first, then each holder's whole step with the exchange replaced by the
+    stack of those partial sums.  Every holder must arrive at bit-identical row statistics,
+    sums, freshness and loss; the gradient is assembled from the holders' column ranges."""
+    def run(chunks_dev, B, tau, H, d_sup=None, params=PARAMS, use_row_ws=True, vocab=None, want_rows=True):
+        dev = chunks_dev[0]["student"].device
+        V = vocab or chunks_dev[0]["student"].shape[1]
+        assert cuts[0] == 0 and cuts[-1] == V
+        p = fb.params(**params)
+        tau_d = torch.as_tensor(np.asarray(tau, dtype=np.int32), device=dev)
+        H_d = torch.as_tensor(np.asarray(H, dtype=np.int32), device=dev)
+        ds_d = None if d_sup is None else torch.as_tensor(np.asarray(d_sup, dtype=np.float32), device=dev)
+        dlogits = [torch.full_like(c["student"], float("nan")) for c in chunks_dev]
+        ranges = list(zip(cuts[:-1], cuts[1:]))
+
+        def shard(c, a, b):
+            return fb.Chunk(c["student"][:, a:b], c["teacher"][:, a:b], c["behav_logprob"], c["tokens"], c["mask"],
+                            c["sample_id"])
+
+        parts = []
+        for c in chunks_dev:
+            n = c["tokens"].numel()
+            stack = torch.empty((len(ranges), n, 8), dtype=torch.float32, device=dev)
+            for k, (a, b) in enumerate(ranges):
+                fb.fopd_shard_stats(shard(c, a, b), a, V, stack[k])
+            parts.append(stack)
+        results = []
+        for k, (a, b) in enumerate(ranges):
+            buf = pl.BatchBuffers(B, dev)
+            rows = [pl.RowOutputs.alloc(c["student"].shape[0], dev) for c in chunks_dev]
+            it = iter(parts)
+            own = []
+
+            def gather(part, it=it, k=k, own=own):
+                stack = next(it)
+                assert torch.equal(part, stack[k])  # this holder's own sums are reproducible
+                return stack
+
+            pl.step_vocab_sharded([shard(c, a, b) for c in chunks_dev], a, V, [d[:, a:b] for d in dlogits], buf,
+                                  tau_d, H_d, ds_d, p, rows, gather=gather)
+            results.append((buf, rows))
+        buf0, rows0 = results[0]
+        for buf, rows in results[1:]:
+            for name in ("acc", "loss_acc", "f", "w", "coef", "loss", "per_sample_loss", "status"):
+                assert torch.equal(getattr(buf, name), getattr(buf0, name)), name
+            for r, r0 in zip(rows, rows0):
+                assert torch.equal(r.row_ws, r0.row_ws) and torch.equal(r.lp_s, r0.lp_s)
+        return buf0, rows0, dlogits, fb.fopd_check_status(buf0.status)
+    return run
+
+
 def compare(chunks_dev, B, tau, H, d_sup=None, params=PARAMS, use_row_ws=True, grad_rows_per_chunk=None,
-            seed=0, expect_bits=0, vocab=None):
+            seed=0, expect_bits=0, vocab=None, runner=None):
     """Full comparison of one batch; returns a dict of the maxima seen."""
-    buf, rows, dlogits, bits = gpu_run(chunks_dev, B, tau, H, d_sup, params, use_row_ws, vocab)
+    buf, rows, dlogits, bits = (runner or gpu_run)(chunks_dev, B, tau, H, d_sup, params, use_row_ws, vocab)
     assert bits == expect_bits, f"device status bits {bits}"
     V = vocab or chunks_dev[0]["student"].shape[1]
     hc = [host_chunk(c) for c in chunks_dev]
