@@ -53,6 +53,8 @@ def parse_args():
     ap.add_argument("--path", default="cached", choices=["cached", "standalone"])
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--vocab-shards", type=int, default=8,
+                    help="also time the vocabulary-sharded entry points with this many column ranges (0: skip)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-on-chip", action="store_true", help="skip the extra timing of the on-chip fwd+bwd kernel")
     ap.add_argument("--cpu-sample-rows", type=int, default=0, help="rows of the CPU-oracle sample (0 = auto)")
@@ -304,6 +306,13 @@ def main():
         torch.cuda.synchronize()
         on_chip_ms = t_begin.elapsed_time(t_end) / args.steps / len(chunks)
 
+    # the vocabulary-sharded entry points on the same rows: every holder's column range in turn
+    # on this one GPU (partial sums of all parts, one merge, every part's gradient), so the sums
+    # over the parts compare with the whole-row kernels above
+    sharded = None
+    if cached and args.vocab_shards > 1 and len(chunks) == 1:
+        sharded = time_vocab_sharded(args, wl, chunks_d[0], dlogits[0], rows[0], buf, p, dev)
+
     coef = buf.coef.cpu().numpy()
     active_rows = int(((coef[np.clip(wl.sample_id, 0, wl.B - 1)] > 0) & (wl.mask > 0)).sum())
     aligned = int(wl.mask.sum())
@@ -349,6 +358,11 @@ def main():
         "clocks": clocks,
         "loss": float(buf.loss.cpu()[0]),
     }
+    if sharded:
+        e = 2 if wl.dtype == torch.bfloat16 else 4
+        sharded["stats_gbs"] = stats_bytes / (sharded["stats_ms_all_parts"] * 1e-3) / 1e9
+        sharded["grad_gbs"] = grad_bytes / (sharded["grad_ms_all_parts"] * 1e-3) / 1e9
+        line["vocab_sharded"] = sharded
 
     # ---- end to end through the host-buffer entry point (pinned host memory, copies timed)
     if not args.no_e2e and len(chunks) >= 1:
@@ -364,6 +378,46 @@ def main():
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def time_vocab_sharded(args, wl, ch, dlogits, row_out, buf, p, dev):
+    """CUDA-event times of fopd_shard_stats (all parts), fopd_shard_merge and
+    fopd_shard_loss_fwd_bwd (all parts) on one chunk; buf.coef holds the step's weights."""
+    import torch
+    from paper_2605_17862_b200 import binding as fb
+
+    K, V, n = args.vocab_shards, wl.V, ch["tokens"].numel()
+    per = 16 // (2 if wl.dtype == torch.bfloat16 else 4)
+    cuts = [0] + [per * ((V * k // K) // per) for k in range(1, K)] + [V]
+    ranges = list(zip(cuts[:-1], cuts[1:]))
+    mk = lambda a, b: fb.Chunk(ch["student"][:, a:b], ch["teacher"][:, a:b], ch["behav_logprob"], ch["tokens"],
+                               ch["mask"], ch["sample_id"])
+    shards = [mk(a, b) for a, b in ranges]
+    parts = torch.empty((K, n, 8), dtype=torch.float32, device=dev)
+    acc = torch.zeros((wl.B, 4), dtype=torch.float64, device=dev)
+    lacc = torch.zeros((wl.B, 2), dtype=torch.float64, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    tot = [0.0, 0.0, 0.0]
+    for it in range(3 + args.steps):
+        ev[0].record()
+        for k, (a, b) in enumerate(ranges):
+            fb.fopd_shard_stats(shards[k], a, V, parts[k])
+        ev[1].record()
+        fb.fopd_shard_merge(parts, ch["behav_logprob"], ch["tokens"], ch["mask"], ch["sample_id"], V, wl.B, acc,
+                            row_out.row_ws, status=status)
+        ev[2].record()
+        for k, (a, b) in enumerate(ranges):
+            fb.fopd_shard_loss_fwd_bwd(shards[k], a, V, wl.B, buf.coef, row_out.row_ws, p, dlogits[:, a:b],
+                                       loss_acc=lacc if k == 0 else None)
+        ev[3].record()
+        torch.cuda.synchronize()
+        if it >= 3:
+            for q in range(3):
+                tot[q] += ev[q].elapsed_time(ev[q + 1]) / args.steps
+    assert fb.fopd_check_status(status) == 0
+    return {"parts": K, "columns_per_part": cuts[1], "stats_ms_all_parts": tot[0], "merge_ms": tot[1],
+            "grad_ms_all_parts": tot[2], "launches_per_pass": 2 * K + 3}
 
 
 def run_e2e(args, wl, chunks_d, dev, world, aligned):
