@@ -65,7 +65,19 @@ def _oracle_measurement(wl):
     return _ORACLE_CACHE[wl.name]
 
 
-def _run_full_size(wl, use_row_ws):
+def _shard_cuts(wl, parts):
+    per = 8 if wl.dtype == torch.bfloat16 else 4  # columns per 16 bytes
+    return [0] + [per * ((wl.V * k // parts) // per) for k in range(1, parts)] + [wl.V]
+
+
+def _shards(ch, cuts):
+    return [(a, fb.Chunk(ch["student"][:, a:b], ch["teacher"][:, a:b], ch["behav_logprob"], ch["tokens"], ch["mask"],
+                         ch["sample_id"])) for a, b in zip(cuts[:-1], cuts[1:])]
+
+
+def _run_full_size(wl, use_row_ws, vocab_parts=0):
+    """vocab_parts > 1: the same comparison through the vocabulary-sharded entry points, all
+    holders played in turn on the one GPU."""
     P = par.PARAMS
     p = fb.params(**P)
     B = wl.B
@@ -82,7 +94,16 @@ def _run_full_size(wl, use_row_ws):
     for j in range(wl.n_chunks):
         ch = synth.gen_chunk(wl, j, DEV)
         r = pl.RowOutputs.alloc(ch["student"].shape[0], DEV)
-        pl.measure([pl.to_chunk(ch)], buf, [r], keep_row_ws=True)
+        if vocab_parts > 1:
+            shards = _shards(ch, _shard_cuts(wl, vocab_parts))
+            parts = torch.empty((len(shards), ch["tokens"].numel(), 8), dtype=torch.float32, device=DEV)
+            for k, (a, sh) in enumerate(shards):
+                fb.fopd_shard_stats(sh, a, wl.V, parts[k])
+            fb.fopd_shard_merge(parts, ch["behav_logprob"], ch["tokens"], ch["mask"], ch["sample_id"], wl.V, B,
+                                buf.acc, r.row_ws, lp_s=r.lp_s, lp_t=r.lp_t, kl=r.kl, ratio=r.ratio,
+                                status=buf.status)
+        else:
+            pl.measure([pl.to_chunk(ch)], buf, [r], keep_row_ws=True)
         st = stats_o[j]
         g = {k: getattr(r, k).cpu().numpy().astype(np.float64) for k in ("lp_s", "lp_t", "kl", "ratio")}
         valid = st.valid.astype(bool)
@@ -134,8 +155,13 @@ def _run_full_size(wl, use_row_ws):
     for j in range(wl.n_chunks):
         ch = synth.gen_chunk(wl, j, DEV)
         dl = torch.full_like(ch["student"], float("nan"))
-        fb.fopd_loss_fwd_bwd(pl.to_chunk(ch), B, buf.coef, p, dl, buf.loss_acc,
-                             row_ws=rows_out[j].row_ws if use_row_ws else None, status=buf.status)
+        if vocab_parts > 1:
+            for k, (a, sh) in enumerate(_shards(ch, _shard_cuts(wl, vocab_parts))):
+                fb.fopd_shard_loss_fwd_bwd(sh, a, wl.V, B, buf.coef, rows_out[j].row_ws, p,
+                                           dl[:, a:a + sh.student.shape[1]], loss_acc=buf.loss_acc if k == 0 else None)
+        else:
+            fb.fopd_loss_fwd_bwd(pl.to_chunk(ch), B, buf.coef, p, dl, buf.loss_acc,
+                                 row_ws=rows_out[j].row_ws if use_row_ws else None, status=buf.status)
         lo, hi = wl.chunk_range(j)
         active = torch.as_tensor((wl.mask[lo:hi] > 0) & (coef[wl.sample_id[lo:hi]] > 0), device=DEV)
         if (~active).any():
@@ -181,6 +207,46 @@ def _run_full_size(wl, use_row_ws):
 def test_reasoning_full_size(use_row_ws):
     wl = synth.reasoning()  # 32,768 x 151,936 bf16: the workload bench.py times
     print(wl.name, wl.n_rows, wl.V, _run_full_size(wl, use_row_ws))
+
+
+def test_reasoning_full_size_vocab_sharded():
+    wl = synth.reasoning()  # eight holders of 18,992 columns each, row pitch 151,936
+    print(wl.name, wl.n_rows, wl.V, _run_full_size(wl, True, vocab_parts=8))
+
+
+def test_reasoning_full_size_from_host_buffers():
+    """fopd_step_host on the benchmark workload: per-sample outputs and the loss against the
+    oracle's measurement over every row, the gradient on the oracle's sampled rows, zeros on
+    every row that is not differentiated."""
+    wl = synth.reasoning()
+    P = par.PARAMS
+    stats_o, picks, subs, acc_o = _oracle_measurement(wl)
+    fr = orc.sample_freshness(acc_o, wl.tau, wl.H, None, P["alpha"], P["beta"], P["xi"])
+    loss_o, per_o = orc.loss(fr, P["lam"])
+    host = [{k: v.cpu().pin_memory() for k, v in synth.gen_chunk(wl, j, DEV).items()} for j in range(wl.n_chunks)]
+    hchunks = [pl.to_chunk(c) for c in host]
+    dl = [torch.full_like(c["student"], float("nan")).pin_memory() for c in host]
+    ws = torch.empty(fb.fopd_step_host_workspace_bytes(hchunks, wl.B, True), dtype=torch.uint8, device=DEV)
+    res = fb.fopd_step_host(hchunks, wl.B, torch.as_tensor(wl.tau), torch.as_tensor(wl.H), None, fb.params(**P), dl,
+                            ws)
+    assert int(res["status_bits"][0]) == 0
+    ok = fr.valid.astype(bool)
+    rel = lambda a, b: (np.abs(a.numpy().astype(np.float64) - b) / np.maximum(np.abs(b), 1e-2))[ok].max()
+    assert max(rel(res["f"], fr.f), rel(res["d_roll"], fr.D_roll), rel(res["l_distill"], fr.ell),
+               rel(res["m_align"], fr.m), rel(res["w"], fr.w)) <= par.TOL_REL
+    assert abs(float(res["loss"][0]) - loss_o) <= par.TOL_REL * max(abs(loss_o), 1e-2)
+    assert (np.abs(res["per_sample_loss"].numpy() - per_o) <= par.TOL_REL * np.maximum(np.abs(per_o), 1e-2)).all()
+    for j, c in enumerate(host):
+        lo, hi = wl.chunk_range(j)
+        active = torch.as_tensor((wl.mask[lo:hi] > 0) & (fr.coef[wl.sample_id[lo:hi]] > 0))
+        z = dl[j][~active].view(torch.int16)  # +0 exactly: all bits clear
+        assert int(z.abs().max()) == 0
+        sel, sub = picks[j], subs[j]
+        g_ref = orc.grad_rows(sub["student"], sub["teacher"], sub["tokens"], sub["behav_logprob"], sub["mask"],
+                              sub["sample_id"], fr.coef, P["lam"], np.arange(len(sel)))
+        g = dl[j][torch.as_tensor(sel)].double().numpy()
+        assert np.isfinite(g).all() and np.abs(g - g_ref).max() <= par.TOL_GRAD_ABS
+        assert bool(torch.isfinite(dl[j]).all()), "a gradient row was never written"
 
 
 @pytest.mark.parametrize("name,use_row_ws", [("tool_use", True), ("coding_agent", False)])
