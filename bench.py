@@ -35,19 +35,27 @@ UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, as a
-# ratio to its algorithmic bytes, from the ncu capture of the 4,096 x 151,936 case summarised in
-# profiles/stream_kernels_4096x151936.md (3.6970 GB measured / 3.7340 GB algorithmic; traffic
-# grows in proportion to the rows, so a full launch is this ratio times its algorithmic bytes).
-# None for kernels that changed since their counters were taken.
-NCU_TRAFFIC_RATIO = {"grad_stream_kernel": 0.9901, "fused_cluster_kernel": 0.9902}
-
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel.
+# grad_stream_kernel: one-pass ncu captures of the workloads themselves (the three counters
+# below take a single pass, so nothing is saved or restored around the launch), summarised in
+# profiles/dram_counters_reasoning_and_config5.md.  fused_cluster_kernel: ratio to its
+# algorithmic bytes from the --set full capture of the 4,096 x 151,936 case
+# (profiles/fused_cluster_kernel_4096x151936.md); its traffic grows in proportion to the rows.
+# A kernel that has changed since its counters were taken is taken out of these tables.
+NCU_TRAFFIC_BYTES = {"grad_stream_kernel": {
+    "reasoning": 23291203584,
+    "roofline_4096x32000": 750339072, "roofline_4096x128256": 3112811264, "roofline_4096x151936": 3696975000,
+    "roofline_16384x32000": 3100727552, "roofline_16384x128256": 12566571520,
+    "roofline_16384x151936": 14895170304, "roofline_65536x32000": 12531350016,
+    "roofline_65536x128256": 50385596928, "roofline_65536x151936": 59700596480,
+}}
+NCU_TRAFFIC_RATIO = {"fused_cluster_kernel": 0.9902}
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="fopd", choices=["fopd", "reference"])
     ap.add_argument("--workload", default="reasoning")
     ap.add_argument("--path", default="cached", choices=["cached", "standalone"])
@@ -184,7 +192,18 @@ def run_reference(args, rank: int):
     print(json.dumps(line), flush=True)
 
 
-def time_oracle(wl, sample_rows: int, steps: int = 1, warmup: int = 0, chunk0=None):
+def cpu_model() -> str:
+    try:
+        with open("/proc/cpuinfo") as fh:
+            for ln in fh:
+                if ln.lower().startswith("model name"):
+                    return ln.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
+def time_oracle(wl, sample_rows: int, steps: int = 1, warmup: int = 0, chunk0=None, threads: int = 0):
     """Times the oracle, as it stands, on the first `sample_rows` aligned rows of
     chunk 0: the statistics pass, per-sample sums, freshness, loss and the
     gradient of every sampled row (the same steps the GPU path runs).  The rows
@@ -205,6 +224,9 @@ def time_oracle(wl, sample_rows: int, steps: int = 1, warmup: int = 0, chunk0=No
                              wl.sigma_s, wl.boost_frac, wl.boost, wl.sigma_t, wl.sigma_b, wl.seed)
         ch = synth.gen_chunk(sub, 0, "cpu", row_block=64)
     P = synth.DEFAULT_PARAMS
+    all_threads = orc.num_threads()
+    if threads:
+        orc.set_threads(threads)
     times = []
     for it in range(warmup + steps):
         t0 = time.perf_counter()
@@ -215,7 +237,10 @@ def time_oracle(wl, sample_rows: int, steps: int = 1, warmup: int = 0, chunk0=No
         if it >= warmup:
             times.append(time.perf_counter() - t0)
     dt = sum(times) / len(times)
-    return {"value": len(aligned) / dt, "ms_per_step": dt * 1e3, "cores": orc.num_threads(),
+    cores = orc.num_threads()
+    if threads:
+        orc.set_threads(all_threads)
+    return {"value": len(aligned) / dt, "ms_per_step": dt * 1e3, "cores": cores,
             "sample": f"first {len(aligned)} aligned rows of chunk 0 ({n} rows incl. masked), V={wl.V}, "
                       f"stats + freshness + loss + gradient of every sampled row, {dt:.1f} s per pass"}
 
@@ -288,8 +313,9 @@ def main():
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     total_ms = t_begin.elapsed_time(t_end)
-    stats_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in events) / len(chunks)
-    grad_ms = statistics.mean(e[2].elapsed_time(e[3]) for e in events) / len(chunks)
+    stats_all = [e[0].elapsed_time(e[1]) / len(chunks) for e in events]
+    grad_all = [e[2].elapsed_time(e[3]) / len(chunks) for e in events]
+    stats_ms, grad_ms = statistics.mean(stats_all), statistics.mean(grad_all)
 
     # the same loss forward + backward without cached row statistics (on-chip kernel), timed
     # on its own after the step timing: what a caller pays when the student logits changed
@@ -325,6 +351,12 @@ def main():
     grad_kernel = "grad_stream_kernel" if cached else (
         "fused_cluster_kernel" if plan["cluster_size"] else "token_stats_kernel+grad_stream_kernel")
     achieved = grad_bytes / n_launch_chunk / (grad_ms * 1e-3) / 1e9
+    traffic, traffic_src = None, None
+    if n_launch_chunk == 1 and wl.name in NCU_TRAFFIC_BYTES.get(grad_kernel, {}):
+        traffic, traffic_src = NCU_TRAFFIC_BYTES[grad_kernel][wl.name], "ncu, one-pass capture of this workload"
+    elif grad_kernel in NCU_TRAFFIC_RATIO and wl.V == 151936:
+        traffic = NCU_TRAFFIC_RATIO[grad_kernel] * grad_bytes / n_launch_chunk
+        traffic_src = "ncu, 4,096-row case of the same kernel scaled by rows"
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -340,6 +372,8 @@ def main():
         },
         "gpu_launches": kernels_per_step * args.steps,
         "phases_ms": {"token_stats_per_chunk": stats_ms, "loss_fwd_bwd_per_chunk": grad_ms,
+                      "token_stats_median_best": [statistics.median(stats_all), min(stats_all)],
+                      "loss_fwd_bwd_median_best": [statistics.median(grad_all), min(grad_all)],
                       "freshness": statistics.mean(e[1].elapsed_time(e[2]) for e in events)},
         "token_stats": {"gbs": stats_bytes / n_launch_chunk / (stats_ms * 1e-3) / 1e9,
                         "frac_of_peak": stats_bytes / n_launch_chunk / (stats_ms * 1e-3) / 1e9 / peak},
@@ -351,9 +385,7 @@ def main():
             "frac_of_peak": grad_bytes / n_launch_chunk / (on_chip_ms * 1e-3) / 1e9 / peak, "plan": plan},
         "roofline": {"bound": "hbm", "kernel": grad_kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": peak_src,
-                     "traffic": (NCU_TRAFFIC_RATIO[grad_kernel] * grad_bytes / n_launch_chunk
-                                 if grad_kernel in NCU_TRAFFIC_RATIO and wl.V == 151936 else None),
-                     "traffic_source": "ncu, 4,096-row case of the same kernel scaled by rows",
+                     "traffic": traffic, "traffic_source": traffic_src,
                      "algorithmic_bytes_per_launch": grad_bytes / n_launch_chunk},
         "clocks": clocks,
         "loss": float(buf.loss.cpu()[0]),
@@ -372,8 +404,10 @@ def main():
             line["e2e"] = {"value": None, "unit": UNIT, "error": repr(exc)[:200]}
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         res = time_oracle(wl, args.cpu_sample_rows or 32768, chunk0=chunks_d[0])
+        one = time_oracle(wl, max(64, (args.cpu_sample_rows or 32768) // 24), chunk0=chunks_d[0], threads=1)
         line["cpu_baseline"] = {"value": res["value"], "unit": UNIT, "cores": res["cores"], "kind": "oracle",
-                                "sample": res["sample"]}
+                                "sample": res["sample"], "cpu_model": cpu_model(), "host_cores": os.cpu_count(),
+                                "single_thread": {"value": one["value"], "sample": one["sample"]}}
     if rank == 0:
         print(json.dumps(line), flush=True)
     if world > 1:
