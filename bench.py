@@ -54,7 +54,7 @@ NCU_TRAFFIC_RATIO = {"fused_cluster_kernel": 0.9902}
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="fopd", choices=["fopd", "reference"])
     ap.add_argument("--workload", default="reasoning")
@@ -100,7 +100,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
                  "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -109,9 +109,10 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([x.strip() for x in line.split(",")])
+            self.rows.append((time.time(), [x.strip() for x in line.split(",")]))
 
-    def stop(self):
+    def stop(self, t0=None, t1=None):
+        """Summary of the samples taken between wall-clock times t0 and t1 (all samples if none fall there)."""
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -121,7 +122,8 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        inside = [r for t, r in self.rows if t0 is not None and t0 <= t <= t1 + 0.05]
+        for r in inside or [r for _, r in self.rows]:
             try:
                 sm.append(float(r[0]))
                 mx.append(float(r[1]))
@@ -132,7 +134,8 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+                "power_w_max": max(pw) if pw else None, "samples": len(sm),
+                "sampled": "during the timed region" if inside else "around the timed region", "reasons": sorted(reasons)}
 
 
 def max_over_ranks(value: float, device=None) -> float:
@@ -269,6 +272,11 @@ def main():
 
     wl = make_workload(args.workload)
     wl.seed = wl.seed + 100 * rank  # independent replica per rank
+    need_dev = 3 * wl.n_rows * wl.V * (2 if wl.dtype == torch.bfloat16 else 4)
+    free_dev, _ = torch.cuda.mem_get_info(dev)
+    if need_dev > 0.9 * free_dev:
+        raise SystemExit("workload %s needs %.0f GB resident (S, T, dlogits of every chunk); %.0f GB free"
+                         % (wl.name, need_dev / 1e9, free_dev / 1e9))
     chunks_d = [synth.gen_chunk(wl, j, dev) for j in range(wl.n_chunks)]
     chunks = [pl.to_chunk(c) for c in chunks_d]
     dlogits = [torch.empty_like(c["student"]) for c in chunks_d]
@@ -306,12 +314,13 @@ def main():
         sampler.start()
         time.sleep(0.3)
     barrier()
+    wall0 = time.time()
     t_begin.record()
     for k in range(args.steps):
         one_step(events[k])
     t_end.record()
     barrier()
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(wall0, time.time()) if rank == 0 else None
     total_ms = t_begin.elapsed_time(t_end)
     stats_all = [e[0].elapsed_time(e[1]) / len(chunks) for e in events]
     grad_all = [e[2].elapsed_time(e[3]) / len(chunks) for e in events]
@@ -399,6 +408,11 @@ def main():
     # ---- end to end through the host-buffer entry point (pinned host memory, copies timed)
     if not args.no_e2e and len(chunks) >= 1:
         try:
+            import psutil
+            need_host = 3 * sum(c["student"].numel() * c["student"].element_size() for c in chunks_d)
+            if need_host > 0.8 * psutil.virtual_memory().available:
+                raise MemoryError("pinned host copies of the batch (%.0f GB) would not fit comfortably in host memory"
+                                  % (need_host / 1e9))
             line["e2e"] = run_e2e(args, wl, chunks_d, dev, world, aligned)
         except Exception as exc:  # report, never fake
             line["e2e"] = {"value": None, "unit": UNIT, "error": repr(exc)[:200]}
