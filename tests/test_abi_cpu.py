@@ -101,6 +101,39 @@ def test_more_host_checks(lib):
     assert lib.fopd_step_host_workspace_bytes((fb.fopd_chunk * 1)(_chunk(dtype=9)), 1, 4, 0) == 0
 
 
+def test_shard_entry_points_check_arguments_on_the_host(lib):
+    vp = ctypes.c_void_p
+    p = fb.params()
+    sh = _chunk(vocab=32, row_stride=64)  # columns [v0, v0 + 32) of rows with a pitch of 64
+    part, ws, coef, acc, out = vp(0x7000), vp(0x8000), vp(0x9000), vp(0xa000), vp(0x100000)
+    assert lib.fopd_shard_stats(ctypes.byref(sh), -8, 64, part, None) == -3            # negative offset
+    assert lib.fopd_shard_stats(ctypes.byref(sh), 40, 64, part, None) == -3            # reaches past the vocabulary
+    assert lib.fopd_shard_stats(ctypes.byref(sh), 0, (1 << 30) + 1, part, None) == -3
+    assert lib.fopd_shard_stats(ctypes.byref(sh), 0, 64, None, None) == -1
+    assert lib.fopd_shard_stats(ctypes.byref(sh), 0, 64, vp(0x7004), None) == -2
+    assert lib.fopd_shard_stats(ctypes.byref(_chunk(student=0x1008, vocab=32)), 0, 64, part, None) == -2
+    assert lib.fopd_shard_stats(None, 0, 64, part, None) == -1
+    assert lib.fopd_shard_stats(ctypes.byref(_chunk(n_rows=0, student=0, teacher=0, vocab=32)), 0, 64, None, None) == 0
+    rows = _chunk(student=0, teacher=0, vocab=64)  # the merge ignores the logits pointers
+    assert lib.fopd_shard_merge(part, 0, ctypes.byref(rows), 2, None, None, None, None, ws, acc, None, None) == -3
+    assert lib.fopd_shard_merge(part, 2, ctypes.byref(rows), 2, None, None, None, None, None, acc, None, None) == -1
+    assert lib.fopd_shard_merge(part, 2, ctypes.byref(rows), 2, None, None, None, None, ws, None, None, None) == -1
+    assert lib.fopd_shard_merge(None, 2, ctypes.byref(rows), 2, None, None, None, None, ws, acc, None, None) == -1
+    assert lib.fopd_shard_merge(part, 2, ctypes.byref(_chunk(tokens=0)), 2, None, None, None, None, ws, acc, None,
+                                None) == -1
+    assert lib.fopd_shard_merge(part, 2, ctypes.byref(rows), 0, None, None, None, None, ws, acc, None, None) == -3
+    assert lib.fopd_shard_merge(part, 2, ctypes.byref(rows), 2, None, None, None, None, vp(0x8004), acc, None,
+                                None) == -2
+    f = lib.fopd_shard_loss_fwd_bwd
+    assert f(ctypes.byref(sh), 0, 64, 2, coef, None, p, out, None, None) == -1        # merged statistics required
+    assert f(ctypes.byref(sh), 0, 64, 2, None, ws, p, out, None, None) == -1
+    assert f(ctypes.byref(sh), 0, 64, 2, coef, ws, p, None, None, None) == -1
+    assert f(ctypes.byref(sh), 40, 64, 2, coef, ws, p, out, None, None) == -3
+    assert f(ctypes.byref(sh), 0, 64, 0, coef, ws, p, out, None, None) == -3
+    assert f(ctypes.byref(sh), 0, 64, 2, coef, ws, fb.params(alpha=-1), out, None, None) == -5
+    assert f(ctypes.byref(sh), 0, 64, 2, coef, ws, p, vp(0x1010), None, None) == -7     # over the student's columns
+
+
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(fb, "_lib", None)
     monkeypatch.setattr(fb, "LIB_PATH", str(tmp_path / "libfopd.so"))
