@@ -125,7 +125,7 @@ def compare(chunks_dev, B, tau, H, d_sup=None, params=PARAMS, use_row_ws=True, g
         r = rows[j]
         valid = st.valid.astype(bool)
         g = {k: getattr(r, k).cpu().numpy().astype(np.float64) for k in ("lp_s", "lp_t", "kl", "ratio")}
-        ws = r.row_ws.cpu().numpy().astype(np.float64)
+        ws = r.row_ws.cpu().numpy().astype(np.float64) if use_row_ws else None  # not written otherwise
         for k in g:  # mask handling is exact: not-aligned rows are exactly zero
             assert np.all(g[k][~valid] == 0.0), k
         if use_row_ws:
