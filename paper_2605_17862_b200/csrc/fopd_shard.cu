@@ -57,9 +57,9 @@ int fopd_shard_merge(const float *partials, int32_t n_parts, const fopd_chunk *r
   int rc = check_rows(rows, B);
   if (rc != FOPD_OK) return rc;
   if (n_parts <= 0) return FOPD_ERR_SIZE;
-  if (!acc || !row_ws) return FOPD_ERR_NULL;
+  if (!acc) return FOPD_ERR_NULL;
   if (rows->n_rows == 0) return FOPD_OK;
-  if (!partials) return FOPD_ERR_NULL;
+  if (!partials || !row_ws) return FOPD_ERR_NULL;
   if (!aligned16(partials) || !aligned16(row_ws)) return FOPD_ERR_ALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const ChunkDev d = to_dev(rows);
@@ -77,9 +77,9 @@ int fopd_shard_loss_fwd_bwd(const fopd_chunk *shard, int64_t vocab_offset, int64
   if (rc != FOPD_OK) return rc;
   if (B <= 0) return FOPD_ERR_SIZE;
   if ((rc = check_params(p)) != FOPD_OK) return rc;
-  if (!coef || !row_ws) return FOPD_ERR_NULL;
+  if (!coef) return FOPD_ERR_NULL;
   if (shard->n_rows == 0) return FOPD_OK;
-  if (!dlogits) return FOPD_ERR_NULL;
+  if (!dlogits || !row_ws) return FOPD_ERR_NULL;
   if (!aligned16(dlogits) || !aligned16(row_ws)) return FOPD_ERR_ALIGN;
   {
     // extents of the three views, from the first column of the first row to the last of the last

@@ -27,7 +27,7 @@ def _run_host(host, B, tau, H, d_sup, params, resident, vocab=None):
     need = fb.fopd_step_host_workspace_bytes(hchunks, B, resident)
     assert need > 0
     if not resident:
-        assert need < fb.fopd_step_host_workspace_bytes(hchunks, B, True) or len(host) == 1
+        assert need <= fb.fopd_step_host_workspace_bytes(hchunks, B, True)
     ws = torch.empty(need, dtype=torch.uint8, device=DEV)
     dl = [torch.full_like(c["student"], float("nan")).pin_memory() for c in host]
     res = fb.fopd_step_host(hchunks, B, torch.as_tensor(np.asarray(tau, np.int32)),

@@ -52,6 +52,14 @@ def test_sharded_uneven_splits_and_tails(dtype, cuts):
     par.compare([ch], B, wl.tau, wl.H, vocab=V, runner=par.gpu_run_vocab_sharded(cuts))
 
 
+def test_sharded_chunks_with_an_empty_one():
+    wl = synth.tiny(scale=1 / 8)
+    ch = synth.gen_chunk(wl, 0, DEV)
+    n = ch["tokens"].numel()
+    chunks = [{k: v[a:b] for k, v in ch.items()} for a, b in ((0, 7), (7, 7), (7, n))]
+    par.compare(chunks, wl.B, wl.tau, wl.H, runner=par.gpu_run_vocab_sharded([0, 8 * (wl.V // 24), wl.V]))
+
+
 def test_partial_sums_match_the_oracle_definition():
     wl = synth.tiny(scale=1 / 8)
     ch = synth.gen_chunk(wl, 0, DEV)
