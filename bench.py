@@ -63,6 +63,9 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--vocab-shards", type=int, default=8,
                     help="also time the vocabulary-sharded entry points with this many column ranges (0: skip)")
+    ap.add_argument("--max-chunks", type=int, default=0,
+                    help="keep only the first K chunks of a chunked workload (0: all; the full tool_use and "
+                         "coding_agent batches hold 134-180 GB on the device)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-on-chip", action="store_true", help="skip the extra timing of the on-chip fwd+bwd kernel")
     ap.add_argument("--cpu-sample-rows", type=int, default=0, help="rows of the CPU-oracle sample (0 = auto)")
@@ -272,6 +275,11 @@ def main():
 
     wl = make_workload(args.workload)
     wl.seed = wl.seed + 100 * rank  # independent replica per rank
+    if args.max_chunks and args.max_chunks < wl.n_chunks:
+        import dataclasses
+        keep = args.max_chunks * wl.chunk_rows
+        wl = dataclasses.replace(wl, name="%s[first %d chunks]" % (wl.name, args.max_chunks),
+                                 sample_id=wl.sample_id[:keep], mask=wl.mask[:keep])
     need_dev = 3 * wl.n_rows * wl.V * (2 if wl.dtype == torch.bfloat16 else 4)
     free_dev, _ = torch.cuda.mem_get_info(dev)
     if need_dev > 0.9 * free_dev:
