@@ -14,6 +14,9 @@ using namespace fopd;
 
 namespace {
 
+// Planning and launching both set per-function attributes of the on-chip kernel: one lock for both.
+std::mutex g_fused_mu;
+
 constexpr int kNotApplicable = 1;  // the on-chip kernel cannot take this shape; use the streaming pair
 
 // Launch shape of the on-chip kernel for one (device, dtype, vocabulary): cluster
@@ -134,11 +137,10 @@ int fused_plan(int64_t nvec, FusedPlan *plan) {
     int64_t nvec;
     FusedPlan plan;
   };
-  static std::mutex mu;
   static std::vector<Entry> cache;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return FOPD_ERR_CUDA;
-  std::lock_guard<std::mutex> lock(mu);
+  std::lock_guard<std::mutex> lock(g_fused_mu);
   for (const Entry &e : cache)
     if (e.dev == dev && e.nvec == nvec) {
       *plan = e.plan;
@@ -163,8 +165,6 @@ int launch_fused(const fopd_chunk *chunk, int32_t B, const float *coef, float la
   if (!plan.cluster || plan.max_clusters < 1) return kNotApplicable;
   const int C = plan.cluster;
   const void *kernel = fused_kernel_for<DT>(plan.threads);
-  // the attributes are per function, and the plan of another vocabulary may have changed them
-  if ((rc = set_fused_attributes(kernel, C, plan.smem)) != FOPD_OK) return rc;
   float *row_cf = tmp + 4 * chunk->n_rows;
   const ChunkDev d = to_dev(chunk);
   row_coef_kernel<<<(unsigned)((chunk->n_rows + 255) / 256), 256, 0, st>>>(d, B, coef, status, row_cf);
@@ -182,6 +182,10 @@ int launch_fused(const fopd_chunk *chunk, int32_t B, const float *coef, float la
   a.status = status;
   a.slice_vecs = plan.slice_vecs;
   void *args[] = {&a};
+  // the attributes are per function, and the plan of another vocabulary may have changed them:
+  // set them and launch under one lock, so that a call from another thread cannot come between
+  std::lock_guard<std::mutex> lock(g_fused_mu);
+  if ((rc = set_fused_attributes(kernel, C, plan.smem)) != FOPD_OK) return rc;
   if (cudaLaunchKernelExC(&cfg, kernel, args) != cudaSuccess) {
     (void)cudaGetLastError();
     return FOPD_ERR_CUDA;

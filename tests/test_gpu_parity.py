@@ -292,6 +292,49 @@ def test_two_streams_run_two_batches_concurrently():
             assert torch.equal(x, y)
 
 
+def test_two_host_threads_with_different_vocabularies():
+    """The on-chip kernel's launch shape depends on the vocabulary and is set per function: two
+    host threads that alternate between two vocabularies on their own streams get the same bits
+    as one thread running them one after the other."""
+    import threading
+
+    wls = [synth.reasoning(scale=1 / 32), synth.reasoning(scale=1 / 8)]  # V = 4,752 and 18,992: different cluster sizes
+    data = [(wl, _chunks(wl)) for wl in wls]
+    refs = [par.gpu_run(ch, wl.B, wl.tau, wl.H, use_row_ws=False) for wl, ch in data]
+    p = fb.params(**par.PARAMS)
+    torch.cuda.synchronize()
+    out, errors = {}, []
+
+    def work(t):
+        try:
+            torch.cuda.set_device(0)
+            s = torch.cuda.Stream(device=DEV)
+            for it in range(6):
+                k = (t + it) % 2
+                wl, ch = data[k]
+                buf = pl.BatchBuffers(wl.B, DEV)
+                dl = [torch.full_like(c["student"], float("nan")) for c in ch]
+                with torch.cuda.stream(s):
+                    pl.step([pl.to_chunk(c) for c in ch], dl, buf, torch.as_tensor(wl.tau, device=DEV),
+                            torch.as_tensor(wl.H, device=DEV), None, p, None, use_row_ws=False, stream=s)
+                s.synchronize()
+                out[(t, it)] = (k, buf, dl)
+        except Exception as exc:  # surfaced below: an exception in a thread would otherwise be lost
+            errors.append(exc)
+
+    threads = [threading.Thread(target=work, args=(t,)) for t in range(2)]
+    for th in threads:
+        th.start()
+    for th in threads:
+        th.join()
+    assert not errors, errors
+    for (t, it), (k, buf, dl) in out.items():
+        assert fb.fopd_check_status(buf.status) == 0
+        assert torch.equal(buf.loss, refs[k][0].loss)
+        for x, y in zip(dl, refs[k][2]):
+            assert torch.equal(x, y)
+
+
 def test_on_chip_plan_is_reported():
     for dtype, V in ((torch.bfloat16, 151936), (torch.bfloat16, 32000), (torch.float32, 32000)):
         plan = fb.fopd_loss_fwd_bwd_plan(dtype, V)
