@@ -184,7 +184,9 @@ def run_reference(args, rank: int):
     from paper_2605_17862_b200 import synth
 
     wl = make_workload(args.workload)
-    res = time_oracle(wl, args.cpu_sample_rows or 2048, steps=args.steps, warmup=args.warmup)
+    # rows per step sized so that warm-up + steps stay within a few minutes on the host cores
+    rows = args.cpu_sample_rows or max(128, min(2048, 40960 // max(1, args.steps + args.warmup)))
+    res = time_oracle(wl, rows, steps=args.steps, warmup=args.warmup)
     line = {
         "impl": "reference", "metric": METRIC, "value": res["value"], "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": res["ms_per_step"], "higher_is_better": True,
