@@ -400,8 +400,8 @@ int fopd_check_status(const int32_t *status, int32_t *bits_out /* HOST */, void 
  *               Otherwise every chunk is uploaded twice (once per phase) and
  *               everything runs on `stream` in order.
  *
- * Host-buffer steps of one process run one at a time (a lock around the shared
- * streams); work queued on `stream` before the call is waited for first.
+ * Host-buffer steps on one device run one at a time (a lock around that device's
+ * shared streams); work queued on `stream` before the call is waited for first.
  * Synchronises `stream` before returning.  Returns FOPD_ERR_SIZE if the
  * workspace is too small, FOPD_ERR_DEVICE if the status word is non-zero (the
  * outputs are still written).

@@ -129,7 +129,7 @@ struct Pipe {
   cudaEvent_t up = nullptr, grad = nullptr, fin = nullptr, slot_free[kMaxSlots] = {};
   bool ok = false;
 };
-std::mutex g_pipe_mu;  // one host-buffer step at a time per process: the pipes are shared state
+std::mutex g_pipe_mu[64];  // one host-buffer step at a time per device: its streams and events are shared state
 Pipe g_pipes[64];
 
 int get_pipe(Pipe **out) {
@@ -176,7 +176,10 @@ int run_pipelined(const fopd_chunk *chunks, const fopd_chunk *dev, int32_t n_chu
                   const float *dsup_d, fopd_params p, float *o_f, float *o_w, float *o_dr, float *o_l, float *o_m,
                   float *o_coef, float *o_means, int32_t *status, void *const *dlogits, UploadRows upload_rows,
                   cudaStream_t st, uint64_t *h2d_bytes) {
-  std::lock_guard<std::mutex> lock(g_pipe_mu);
+  int device = 0;
+  CU(cudaGetDevice(&device));
+  if (device < 0 || device >= 64) return FOPD_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_pipe_mu[device]);
   Pipe *P = nullptr;
   RC(get_pipe(&P));
   const uint64_t R = L.rows_total;
