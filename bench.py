@@ -420,7 +420,8 @@ def main():
         try:
             import psutil
             need_host = 3 * sum(c["student"].numel() * c["student"].element_size() for c in chunks_d)
-            if need_host > 0.8 * psutil.virtual_memory().available:
+            # from the host's total memory, so that every rank takes the same decision
+            if need_host * world > 0.6 * psutil.virtual_memory().total:
                 raise MemoryError("pinned host copies of the batch (%.0f GB) would not fit comfortably in host memory"
                                   % (need_host / 1e9))
             line["e2e"] = run_e2e(args, wl, chunks_d, dev, world, aligned)
