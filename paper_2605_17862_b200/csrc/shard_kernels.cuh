@@ -99,15 +99,16 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads)
   for (int64_t n = blockIdx.x; n < c.n_rows; n += gridDim.x) {
     char *orow = reinterpret_cast<char *>(dlogits) + n * c.stride * E::kBytes;
     const int32_t sid = c.sid[n], y = c.tokens[n];
-    float cf = 0.f;
-    if (c.mask[n] != 0 && sid >= 0 && sid < B && y >= 0 && y < v_total) cf = coef[sid];
+    const uint8_t m = c.mask[n];
+    const float4 ws = reinterpret_cast<const float4 *>(row_ws)[n];
+    float cf = (sid >= 0 && sid < B) ? coef[sid] : 0.f;
+    if (m == 0 || y < 0 || y >= v_total) cf = 0.f;
     if (!(cf > 0.f)) {
       zero_fill_row<DT, kThreads>(orow, c.vocab);
       continue;
     }
     const int64_t yl = (int64_t)y - v0;
-    const GradRow r = make_grad_row(reinterpret_cast<const float4 *>(row_ws)[n], cf, lambda,
-                                    (yl >= 0 && yl < c.vocab) ? (int32_t)yl : -1);
+    const GradRow r = make_grad_row(ws, cf, lambda, (yl >= 0 && yl < c.vocab) ? (int32_t)yl : -1);
     grad_row_sweep<DT, kThreads>(reinterpret_cast<const char *>(c.student) + n * c.stride * E::kBytes,
                                  reinterpret_cast<const char *>(c.teacher) + n * c.stride * E::kBytes, orow, c.vocab,
                                  r);

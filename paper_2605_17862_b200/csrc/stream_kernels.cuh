@@ -33,14 +33,16 @@ struct ChunkDev {
 // Is row n aligned (counts towards U_i)?  Records bad ids in the status word.
 __device__ __forceinline__ bool row_is_aligned(const ChunkDev &c, int64_t n, int32_t B,
                                                int32_t *status, bool report) {
-  const int32_t sid = c.sid[n];
+  // three independent loads, issued together: a CTA's first logits load waits for one memory
+  // round trip, not for a chain of them (tokens[n] is read for masked rows too; it is not used)
+  const int32_t sid = c.sid[n], y = c.tokens[n];
+  const uint8_t m = c.mask[n];
   bool ok = true;
   if (sid < 0 || sid >= B) {
     if (report && status) atomicOr(status, FOPD_DEV_BAD_SAMPLE);
     ok = false;
   }
-  if (c.mask[n] == 0) return false;
-  const int32_t y = c.tokens[n];
+  if (m == 0) return false;
   if (y < 0 || y >= c.vocab) {
     if (report && status) atomicOr(status, FOPD_DEV_BAD_TOKEN);
     ok = false;
@@ -239,13 +241,19 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads)
   using E = Elem<DT>;
   for (int64_t n = blockIdx.x; n < c.n_rows; n += gridDim.x) {
     char *orow = reinterpret_cast<char *>(dlogits) + n * c.stride * E::kBytes;
-    float cf = 0.f;
-    if (row_is_aligned(c, n, B, nullptr, false)) cf = coef[c.sid[n]];
+    // independent loads first (side arrays and cached statistics), then the one that depends
+    // on them (the sample's weight): two memory round trips before the first logits load
+    const int32_t sid = c.sid[n], y = c.tokens[n];
+    const uint8_t m = c.mask[n];
+    const float4 ws = reinterpret_cast<const float4 *>(row_ws)[n];
+    const bool sid_ok = sid >= 0 && sid < B;
+    float cf = sid_ok ? coef[sid] : 0.f;
+    if (m == 0 || y < 0 || y >= c.vocab) cf = 0.f;
     if (!(cf > 0.f)) {
       zero_fill_row<DT, kThreads>(orow, c.vocab);
       continue;
     }
-    const GradRow r = make_grad_row(reinterpret_cast<const float4 *>(row_ws)[n], cf, lambda, c.tokens[n]);
+    const GradRow r = make_grad_row(ws, cf, lambda, y);
     grad_row_sweep<DT, kThreads>(reinterpret_cast<const char *>(c.student) + n * c.stride * E::kBytes,
                                  reinterpret_cast<const char *>(c.teacher) + n * c.stride * E::kBytes, orow, c.vocab,
                                  r);
