@@ -43,11 +43,11 @@ FALLBACK_HBM_GBS = 6650.0
 # (profiles/fused_cluster_kernel_4096x151936.md); its traffic grows in proportion to the rows.
 # A kernel that has changed since its counters were taken is taken out of these tables.
 NCU_TRAFFIC_BYTES = {"grad_stream_kernel": {
-    "reasoning": 23291203584,
-    "roofline_4096x32000": 750339072, "roofline_4096x128256": 3112811264, "roofline_4096x151936": 3696975000,
-    "roofline_16384x32000": 3100727552, "roofline_16384x128256": 12566571520,
-    "roofline_16384x151936": 14895170304, "roofline_65536x32000": 12531350016,
-    "roofline_65536x128256": 50385596928, "roofline_65536x151936": 59700596480,
+    "reasoning": 23291478784,
+    "roofline_4096x32000": 750365440, "roofline_4096x128256": 3112168192, "roofline_4096x151936": 3697052000,
+    "roofline_16384x32000": 3101060096, "roofline_16384x128256": 12566872320,
+    "roofline_16384x151936": 14894971136, "roofline_65536x32000": 12529531136,
+    "roofline_65536x128256": 50388422656, "roofline_65536x151936": 59700739072,
 }}
 NCU_TRAFFIC_RATIO = {"fused_cluster_kernel": 0.9902}
 
