@@ -62,23 +62,27 @@ static void fused_launch_config(cudaLaunchConfig_t *cfg, cudaLaunchAttribute *at
   cfg->numAttrs = 1;
 }
 
-// How evenly `threads - 32` compute threads share a slice of `slice` vectors: work done
-// over work slots (1 = every thread sweeps the same number of vectors).
-static double split_efficiency(int64_t slice, int threads) {
+// Estimated SM cycles a cluster spends on one row: a fixed part per row (barrier hand-offs, the
+// merge of the warps' partial sums, the exchange, which grows with the cluster) plus one round
+// per vector a compute thread sweeps in both sweeps, a round costing in proportion to the warps
+// that share the SM's four schedulers.  Constants fitted to timings on B200 at five vocabularies
+// between 32,000 and 151,936 (blocks of 512-1,024 threads, clusters of 2-12).
+static double row_cycles(int64_t slice, int C, int threads, int ctas_per_sm, double pairs_per_vec) {
   const int64_t ct = threads - 32, rounds = (slice + ct - 1) / ct;
-  return rounds ? (double)slice / (double)(ct * rounds) : 0.0;
+  const double per_round = 46.25 * (pairs_per_vec / 8.0) * (double)(threads / 32 - 1) * ctas_per_sm;
+  return 1800.0 + 50.0 * C + (double)rounds * per_round;
 }
 
-// Picks cluster size and block size with three slice buffers per CTA: the pair that keeps
-// the most CTAs resident (how many clusters of a given size fit depends on how the SMs are
-// grouped) weighted by how evenly the block shares its slice; among equals the smaller
-// cluster and the larger block.  FOPD_FUSED_CLUSTER / FOPD_FUSED_THREADS in the environment
-// pin them.
+// Picks cluster size and block size with three slice buffers per CTA: the pair with the most
+// rows per cycle = resident clusters (how many clusters of a given size fit depends on how the
+// SMs are grouped) over the estimated cycles per row; among equals the smaller cluster and the
+// larger block.  FOPD_FUSED_CLUSTER / FOPD_FUSED_THREADS in the environment pin them.
 template <int DT>
 int make_fused_plan(int64_t nvec, FusedPlan *plan) {
-  int dev = 0, max_optin = 0;
+  int dev = 0, max_optin = 0, n_sm = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&max_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess)
+      cudaDeviceGetAttribute(&max_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm < 1)
     return FOPD_ERR_CUDA;
   const size_t fixed = ((sizeof(ClusterShared) + 127) & ~size_t(127));
   const char *pin_c = getenv("FOPD_FUSED_CLUSTER"), *pin_t = getenv("FOPD_FUSED_THREADS");
@@ -94,37 +98,45 @@ int make_fused_plan(int64_t nvec, FusedPlan *plan) {
     const int64_t slice = (nvec + C - 1) / C;
     const size_t smem = fixed + (size_t)kSliceBufs * 2 * (size_t)slice * 16;
     if (smem > (size_t)max_optin || slice * 32 >= (1 << 20)) continue;  // one copy barrier counts < 2^20 bytes
-    int threads = 0;
-    double eff = 0.0;
-    for (int t : choices) {
-      if (pin_t && atoi(pin_t) != t) continue;
-      const double e = split_efficiency(slice, t);
-      if (e >= eff) {
-        eff = e;
-        threads = t;
+    for (int threads : choices) {
+      if (pin_t && atoi(pin_t) != threads) continue;
+      const void *kernel = fused_kernel_for<DT>(threads);
+      int rc = set_fused_attributes(kernel, C, smem);
+      if (rc != FOPD_OK) return rc;
+      cudaLaunchConfig_t cfg;
+      cudaLaunchAttribute attr[1];
+      fused_launch_config(&cfg, attr, C, threads, smem, (unsigned)C, nullptr);
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) {
+        (void)cudaGetLastError();
+        n = 0;
+      }
+      if (n < 1) continue;
+      const int ctas_per_sm = (n * C + n_sm - 1) / n_sm;
+      const double score = (double)n / row_cycles(slice, C, threads, ctas_per_sm, Elem<DT>::kPerVec);
+      if (score >= best_score * 1.0001 || (score > best_score * 0.9999 && C == best.cluster)) {
+        best_score = score > best_score ? score : best_score;
+        best.cluster = C;
+        best.threads = threads;
+        best.slice_vecs = (int)slice;
+        best.smem = smem;
+        best.max_clusters = n;
       }
     }
-    if (!threads) continue;
-    const void *kernel = fused_kernel_for<DT>(threads);
-    int rc = set_fused_attributes(kernel, C, smem);
-    if (rc != FOPD_OK) return rc;
-    cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attr[1];
-    fused_launch_config(&cfg, attr, C, threads, smem, (unsigned)C, nullptr);
-    int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) {
-      (void)cudaGetLastError();
-      n = 0;
-    }
-    const double score = (double)n * C * eff;
-    if (score > best_score * 1.0001) {
-      best_score = score;
-      best.cluster = C;
-      best.threads = threads;
-      best.slice_vecs = (int)slice;
-      best.smem = smem;
-      best.max_clusters = n;
-    }
+  }
+  // Against the two streaming sweeps, which move five thirds of the bytes at ~80 % of the
+  // memory system's nominal rate: very long rows leave too few clusters resident for the
+  // on-chip kernel to win, and then the streaming pair is what runs.
+  int sm_khz = 0, mem_khz = 0, bus_bits = 0;
+  if (best.cluster && !pin_c && !pin_t && nvec >= kShortRowVecs &&  // (short rows: both paths are latency-bound)
+      cudaDeviceGetAttribute(&sm_khz, cudaDevAttrClockRate, dev) == cudaSuccess &&
+      cudaDeviceGetAttribute(&mem_khz, cudaDevAttrMemoryClockRate, dev) == cudaSuccess &&
+      cudaDeviceGetAttribute(&bus_bits, cudaDevAttrGlobalMemoryBusWidth, dev) == cudaSuccess && sm_khz > 0 &&
+      mem_khz > 0 && bus_bits > 0) {
+    const double on_chip_s = 1.0 / (best_score * sm_khz * 1e3);
+    const double bytes_per_s = 0.8 * 2.0 * mem_khz * 1e3 * (bus_bits / 8.0);
+    const double pair_s = 5.0 * (double)nvec * 16.0 / bytes_per_s;
+    if (on_chip_s > pair_s) best = FusedPlan();
   }
   *plan = best;
   return FOPD_OK;

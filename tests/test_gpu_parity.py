@@ -202,8 +202,9 @@ def test_host_validation_errors():
 @pytest.mark.parametrize("V", [40_000, 100_000, 151_936, 300_000, 1_000_000, 40_003])
 def test_standalone_fwd_bwd_across_cluster_sizes(V):
     """fopd_loss_fwd_bwd without cached statistics keeps each row on chip in a
-    thread-block cluster whose size grows with the vocabulary (1, 2, 4, 8 CTAs);
-    a row too large for eight CTAs falls back to the two streaming kernels."""
+    thread-block cluster whose size grows with the vocabulary; rows so long that too few
+    clusters would be resident, or that do not fit sixteen CTAs, go to the two streaming
+    kernels instead."""
     rng = np.random.RandomState(V % 1000)
     B, lengths = 3, np.array([9, 17, 14])
     n = int(lengths.sum())
@@ -215,6 +216,26 @@ def test_standalone_fwd_bwd_across_cluster_sizes(V):
     ch = synth.gen_chunk(wl, 0, DEV, row_block=8, row_stride=stride)
     out = par.compare([ch], B, wl.tau, wl.H, use_row_ws=False, vocab=V, grad_rows_per_chunk=12)
     print(V, out)
+
+
+@pytest.mark.parametrize("V,cluster", [(200_008, 12), (250_008, 16), (60_008, 7), (30_008, 3)])
+def test_on_chip_kernel_with_pinned_cluster_sizes(V, cluster, monkeypatch):
+    """Cluster sizes the planner would not pick for these vocabularies, the non-portable ones
+    (more than eight CTAs) included.  The plan of a vocabulary is made once per process, so each
+    case has a vocabulary of its own."""
+    monkeypatch.setenv("FOPD_FUSED_CLUSTER", str(cluster))
+    plan = fb.fopd_loss_fwd_bwd_plan(torch.bfloat16, V)
+    assert plan["cluster_size"] == cluster and plan["resident_clusters"] >= 1
+    rng = np.random.RandomState(cluster)
+    B, lengths = 3, np.array([9, 17, 14])
+    n = int(lengths.sum())
+    sid = np.repeat(np.arange(B, dtype=np.int32), lengths)
+    mask = (rng.rand(n) > 0.25).astype(np.uint8)
+    wl = synth.Workload("pinned", B, V, torch.bfloat16, n, sid, mask, np.array([0, 1, 2], np.int32),
+                        lengths.astype(np.int32), seed=cluster)
+    ch = synth.gen_chunk(wl, 0, DEV, row_block=8)
+    out = par.compare([ch], B, wl.tau, wl.H, use_row_ws=False, grad_rows_per_chunk=12)
+    print(V, cluster, out)
 
 
 def test_ablation_objectives_are_parameter_settings():
