@@ -231,12 +231,15 @@ int fopd_loss_fwd_bwd(const fopd_chunk *chunk /* HOST */, int32_t B,
  * threads per CTA, clusters resident at once and dynamic shared memory per CTA
  * (three slice buffers: the copies of the row after next overlap the sweeps of
  * the current rows).  All outputs are HOST pointers and may be NULL.
- * *cluster_size = 0 means that no on-chip shape fits (three row pairs do not
- * fit in sixteen CTAs' shared memory) and the call runs the statistics sweep
- * followed by the streaming gradient sweep instead.  The choice is made once
- * per (device, dtype, vocabulary) with cudaOccupancyMaxActiveClusters and
- * cached; the environment variables FOPD_FUSED_CLUSTER and FOPD_FUSED_THREADS,
- * read at that moment, pin it.
+ * *cluster_size = 0 means that the call runs the statistics sweep and the
+ * streaming gradient sweep instead: no on-chip shape fits (three row pairs do
+ * not fit in sixteen CTAs' shared memory), or the row is so long that too few
+ * clusters would be resident for the on-chip kernel to be the faster of the two
+ * (on B200, bf16 rows of about 200,000 logits and more).  The shape is chosen
+ * once per (device, dtype, vocabulary) from cudaOccupancyMaxActiveClusters and
+ * an estimate of the cycles a cluster spends on a row, and cached; the
+ * environment variables FOPD_FUSED_CLUSTER and FOPD_FUSED_THREADS, read when a
+ * vocabulary is first planned, pin the cluster size and the block size.
  */
 int fopd_loss_fwd_bwd_plan(int32_t dtype, int64_t vocab, int32_t *cluster_size,
                            int32_t *block_threads, int32_t *resident_clusters,
