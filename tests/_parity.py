@@ -213,6 +213,12 @@ def compare(chunks_dev, B, tau, H, d_sup=None, params=PARAMS, use_row_ws=True, g
         cf = fr.coef[np.clip(c["sample_id"].numpy()[sel], 0, B - 1)] * st.valid[sel]
         cp = cf[:, None] * np.exp(S64 - st.lse_s[sel, None])
         bound = (out_ulp(dl.dtype) + 2e-5) * np.abs(g_ref) + 2e-5 * cp + 1e-30
+        # the gradient is linear in the sample's weight, which has a tolerance of its own (checked
+        # above): near the gate w = f - xi loses relative accuracy by cancellation, and that much
+        # of the difference belongs to the weight, not to the gradient sweep
+        cf_gpu = buf.coef.cpu().numpy().astype(np.float64)
+        rel_w = np.where(fr.coef > 0, np.abs(cf_gpu - fr.coef) / np.maximum(fr.coef, 1e-300), 0.0)
+        bound += rel_w[np.clip(c["sample_id"].numpy()[sel], 0, B - 1)][:, None] * np.abs(g_ref)
         ycol = np.clip(c["tokens"].numpy()[sel], 0, V - 1)
         # d = lp_s - b carries the absolute fp32 error of the log-normaliser (~1e-6), so the
         # anchor term lambda * rho * d at the stored token has an absolute, not relative, error
