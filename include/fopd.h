@@ -38,11 +38,25 @@
  * pointer to memory the caller owns; the library keeps no pointer after a call
  * returns.  Where a call needs temporary device memory
  * that the caller did not supply (see row_ws) it takes it from a stream-ordered
- * memory pool of its own (one per device, which keeps the memory it has grown
- * to) on the caller's stream and returns it there.  All
+ * memory pool of its own on the caller's stream and returns it there.  All
  * work is enqueued on `stream` (a cudaStream_t passed as void*, NULL = default
  * stream) and the call returns without synchronising, except
- * fopd_check_status.
+ * fopd_check_status and fopd_step_host.
+ *
+ * Process-wide state (all of it; none is read from the environment):
+ *   - one memory pool per device for those temporaries.  It keeps what it has
+ *     grown to (a few bytes per token row of the largest chunk seen) until
+ *     fopd_release_device_memory;
+ *   - the launch shape chosen for fopd_loss_fwd_bwd(row_ws = NULL) per (device,
+ *     dtype, vocabulary), made on first use and cached: fopd_loss_fwd_bwd_plan
+ *     reads it, fopd_loss_fwd_bwd_set_plan sets it;
+ *   - two streams and a few events per device used by fopd_step_host, made on
+ *     its first call, with a lock that lets one host-buffer step run at a time
+ *     per device; fopd_release_device_memory destroys them;
+ *   - the fixed scratch array of fopd_token_stats_static and its cached device
+ *     address per device.
+ * Calls with disjoint buffers may run concurrently from several host threads
+ * and on several streams.
  *
  * Errors.  Every function returns FOPD_OK or a negative fopd_status found on
  * the host before anything is enqueued.  Conditions only visible on the device
@@ -59,7 +73,7 @@
 extern "C" {
 #endif
 
-#define FOPD_VERSION 100
+#define FOPD_VERSION 200
 
 typedef enum { FOPD_BF16 = 0, FOPD_F32 = 1 } fopd_dtype;
 
@@ -164,8 +178,13 @@ int fopd_token_stats(const fopd_chunk *chunk /* HOST */, int32_t B, float *lp_s,
  *   - chunk->n_rows > FOPD_STATIC_MAX_ROWS returns FOPD_ERR_SIZE and enqueues
  *     nothing; split the chunk.
  *   - The first call on each device looks the array's device address up
- *     (cudaGetSymbolAddress, with that device current) and caches it; make
- *     that first call outside any stream capture.
+ *     (cudaGetSymbolAddress, with that device current) and caches it.  With
+ *     CUDA's lazy module loading that first call is also what loads the part of
+ *     the library that holds the array and these kernels onto the device, which
+ *     does reserve device memory once: make the first call on each device
+ *     outside any stream capture and before the rest of the device's memory is
+ *     handed to another allocator.  If it fails it returns FOPD_ERR_CUDA and
+ *     can be repeated.
  *   - All calls on a device share the one array, which still holds the previous
  *     call's values.  Nothing has to be cleared: each call overwrites the
  *     entries of all its rows before it reads them.  Two calls whose kernels can
@@ -229,21 +248,29 @@ int fopd_loss_fwd_bwd(const fopd_chunk *chunk /* HOST */, int32_t B,
  * Launch shape fopd_loss_fwd_bwd(row_ws = NULL) uses on the current device for
  * a vocabulary and dtype: CTAs per thread-block cluster (one cluster per row),
  * threads per CTA, clusters resident at once and dynamic shared memory per CTA
- * (three slice buffers: the copies of the row after next overlap the sweeps of
- * the current rows).  All outputs are HOST pointers and may be NULL.
+ * (three slice buffers that rows' copies land in; the rows being worked on are
+ * held in registers).  All outputs are HOST pointers and may be NULL.
  * *cluster_size = 0 means that the call runs the statistics sweep and the
- * streaming gradient sweep instead: no on-chip shape fits (three row pairs do
- * not fit in sixteen CTAs' shared memory), or the row is so long that too few
- * clusters would be resident for the on-chip kernel to be the faster of the two
- * (on B200, bf16 rows of about 200,000 logits and more).  The shape is chosen
- * once per (device, dtype, vocabulary) from cudaOccupancyMaxActiveClusters and
- * an estimate of the cycles a cluster spends on a row, and cached; the
- * environment variables FOPD_FUSED_CLUSTER and FOPD_FUSED_THREADS, read when a
- * vocabulary is first planned, pin the cluster size and the block size.
+ * streaming gradient sweep instead: no on-chip shape fits (a CTA's slice of a row
+ * must fit its threads' registers: bf16 rows of up to about 295,000 logits in
+ * sixteen CTAs), or the row is so long that fewer than two thirds of the SMs
+ * would hold a resident CTA.  The shape is chosen once per (device, dtype,
+ * vocabulary) from cudaOccupancyMaxActiveClusters -- the cluster size that keeps
+ * the most CTAs resident -- and cached.
  */
 int fopd_loss_fwd_bwd_plan(int32_t dtype, int64_t vocab, int32_t *cluster_size,
                            int32_t *block_threads, int32_t *resident_clusters,
                            int32_t *smem_bytes);
+
+/*
+ * Sets that launch shape for (current device, dtype, vocab) instead of letting
+ * the library choose: cluster_size > 0 pins the CTAs per cluster (FOPD_ERR_SIZE if
+ * a cluster of that size cannot hold a row of this vocabulary on this device,
+ * in which case the plan is left as it was), cluster_size < 0 makes the call
+ * always run the two streaming sweeps, cluster_size = 0 goes back to the
+ * library's own choice.  Takes effect for calls made after it returns.
+ */
+int fopd_loss_fwd_bwd_set_plan(int32_t dtype, int64_t vocab, int32_t cluster_size);
 
 /*
  * After the last chunk: per_sample_loss[i] = w_i (l_i + lambda D_roll_i) with
@@ -370,6 +397,27 @@ int fopd_shard_merge(const float *partials, int32_t n_parts, const fopd_chunk *r
 int fopd_shard_loss_fwd_bwd(const fopd_chunk *shard, int64_t vocab_offset, int64_t vocab_total,
                             int32_t B, const float *coef, const float *row_ws, fopd_params p,
                             void *dlogits, double *loss_acc, void *stream);
+
+/*
+ * Gives back what the library holds on the current device between calls: trims
+ * its memory pool to what pending work still uses and destroys the streams and
+ * events of fopd_step_host (both come back on the next call that needs them).
+ * Waits for a host-buffer step in progress on that device; synchronise the
+ * streams other calls were enqueued on first if all of the pool is to be freed.
+ */
+int fopd_release_device_memory(void);
+
+/*
+ * Self-test of the bounded in-kernel wait.  Every wait on a barrier inside the
+ * library's kernels gives up after a fixed number of SM cycles, records
+ * FOPD_DEV_TIMEOUT in the status word and lets the kernel end.  This call runs
+ * that wait on one CTA against a barrier that is one arrival short, with a
+ * limit of limit_cycles SM cycles (0 <= limit_cycles <= 200,000,000): the wait
+ * must run out, *status gets FOPD_DEV_TIMEOUT and *waited_cycles (DEVICE int64,
+ * may be NULL) the cycles the wait took.  The context stays usable.
+ */
+int fopd_selftest_bounded_wait(int64_t limit_cycles, int32_t *status, int64_t *waited_cycles,
+                               void *stream);
 
 /* Synchronises `stream`, reads the device status word and returns FOPD_OK,
  * FOPD_ERR_DEVICE (word non-zero; *bits_out receives it if not NULL, HOST) or

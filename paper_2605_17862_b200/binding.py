@@ -21,6 +21,7 @@ EXPORTS = (
     "fopd_check_status", "fopd_strerror", "fopd_version", "fopd_step_host", "fopd_step_host_workspace_bytes",
     "fopd_token_stats_static", "fopd_loss_fwd_bwd_plan", "fopd_row_divergence", "fopd_supervision_drift",
     "fopd_refresh_decision", "fopd_shard_stats", "fopd_shard_merge", "fopd_shard_loss_fwd_bwd",
+    "fopd_loss_fwd_bwd_set_plan", "fopd_release_device_memory", "fopd_selftest_bounded_wait",
 )
 
 
@@ -72,6 +73,9 @@ def lib() -> ctypes.CDLL:
         L.fopd_loss_fwd_bwd.argtypes = [ctypes.POINTER(fopd_chunk), i32, vp, vp, fopd_params, vp, vp, vp, vp]
         L.fopd_loss_fwd_bwd_plan.argtypes = [i32, ctypes.c_int64] + [ctypes.POINTER(ctypes.c_int32)] * 4
         i64, f32 = ctypes.c_int64, ctypes.c_float
+        L.fopd_loss_fwd_bwd_set_plan.argtypes = [i32, i64, i32]
+        L.fopd_release_device_memory.argtypes = []
+        L.fopd_selftest_bounded_wait.argtypes = [i64, vp, vp, vp]
         L.fopd_row_divergence.argtypes = [vp, vp, vp, vp, i64, i64, i64, i32, i32, vp, vp, vp, vp, vp]
         L.fopd_supervision_drift.argtypes = [vp, vp, i32, vp, vp, vp, vp]
         L.fopd_refresh_decision.argtypes = [vp, vp, vp, i32, f32, f32, f32, i64, i64, vp, vp, vp]
@@ -196,6 +200,24 @@ def fopd_loss_fwd_bwd_plan(dtype: torch.dtype, vocab: int) -> dict:
                                         *[ctypes.byref(o) for o in out]), "fopd_loss_fwd_bwd_plan")
     return dict(zip(("cluster_size", "block_threads", "resident_clusters", "smem_bytes"),
                     (int(o.value) for o in out)))
+
+
+def fopd_loss_fwd_bwd_set_plan(dtype: torch.dtype, vocab: int, cluster_size: int) -> None:
+    """Pins the on-chip launch shape for (current device, dtype, vocab): cluster_size > 0 CTAs per
+    cluster, < 0 the streaming kernel pair, 0 back to the library's own choice."""
+    _check(lib().fopd_loss_fwd_bwd_set_plan(FOPD_BF16 if dtype == torch.bfloat16 else FOPD_F32, int(vocab),
+                                            int(cluster_size)), "fopd_loss_fwd_bwd_set_plan")
+
+
+def fopd_release_device_memory() -> None:
+    """Trims the library's memory pool on the current device and drops fopd_step_host's streams."""
+    _check(lib().fopd_release_device_memory(), "fopd_release_device_memory")
+
+
+def fopd_selftest_bounded_wait(limit_cycles: int, status, waited_cycles=None, *, stream=None) -> None:
+    """Runs one bounded barrier wait that cannot complete; the kernel sets the timeout bit in ``status``."""
+    _check(lib().fopd_selftest_bounded_wait(int(limit_cycles), _ptr(status), _ptr(waited_cycles), _stream(stream)),
+           "fopd_selftest_bounded_wait")
 
 
 def fopd_loss_finalize(loss_acc, acc, w, B: int, p: fopd_params, loss_out, *, per_sample_loss=None,

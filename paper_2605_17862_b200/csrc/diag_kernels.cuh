@@ -13,11 +13,13 @@ namespace fopd {
 constexpr int kDiagThreads = 256;
 
 // Row accumulators for KL(p || q) and H(p): p-side max m, Z = sum e^{a-m},
-// A = sum e^{a-m} (a - b), S = sum e^{a-m} a; q-side max and Z.
-//   KL = A / Z - lse_p + lse_q,   H(p) = lse_p - S / Z.
+// A = sum e^{a-m} (a - b), S = sum e^{a-m} (a - m); q-side max and Z.
+//   KL = A / Z - lse_p + lse_q,   H(p) = lse_p - E_p[a] = log Z - S / Z.
+// Exponents are formed as (x - max) * log2(e) and the entropy sum is kept relative to the
+// maximum, so neither loses accuracy when the logits sit far from zero.
 struct DivAcc {
   RowAcc r;
-  float ss;  // sum e^{a-m} a, scaled like r.zs
+  float ss;  // sum e^{a-m} (a - m), relative to the same running maximum as r.zs
   __device__ __forceinline__ void init() {
     r.init();
     ss = 0.f;
@@ -26,30 +28,32 @@ struct DivAcc {
   __device__ __forceinline__ void add(const float (&a)[N], const float (&b)[N]) {
     const float va = max_of<N>(a), vb = max_of<N>(b);
     if (va > r.ms) {
+      // new maximum m': sum e^{a-m'} (a - m') = e^{m-m'} (S + (m - m') Z)
       const float f = ex2((r.ms - va) * kLog2e);
+      ss = f * fmaf(r.ms - va, r.zs, ss);
       r.zs *= f;
       r.as *= f;
-      ss *= f;
       r.ms = va;
     }
     if (vb > r.mt) {
       r.zt *= ex2((r.mt - vb) * kLog2e);
       r.mt = vb;
     }
-    const float ba = -r.ms * kLog2e, bb = -r.mt * kLog2e;
 #pragma unroll
     for (int i = 0; i < N; ++i) {
-      const float ea = ex2(fmaf(a[i], kLog2e, ba));
+      const float da = a[i] - r.ms;
+      const float ea = ex2(da * kLog2e);
       r.zs += ea;
       r.as = fmaf(ea, a[i] - b[i], r.as);
-      ss = fmaf(ea, a[i], ss);
-      r.zt += ex2(fmaf(b[i], kLog2e, bb));
+      ss = fmaf(ea, da, ss);
+      r.zt += ex2((b[i] - r.mt) * kLog2e);
     }
   }
   __device__ __forceinline__ void merge(const DivAcc &o) {
     const float M = fmaxf(r.ms, o.r.ms);
     const float fa = ex2((r.ms - M) * kLog2e), fb = ex2((o.r.ms - M) * kLog2e);
-    ss = __fmaf_rn(ss, fa, __fmul_rn(o.ss, fb));
+    // both sums moved to the common maximum M before they are added
+    ss = __fmaf_rn(__fmaf_rn(r.ms - M, r.zs, ss), fa, __fmul_rn(__fmaf_rn(o.r.ms - M, o.r.zs, o.ss), fb));
     r.merge(o.r);
   }
 };
@@ -119,8 +123,8 @@ __global__ void __launch_bounds__(kDiagThreads, 4)
       if (lane == 0) {
         const float gp = logf(t.r.zs), gq = logf(t.r.zt);
         const float kl = t.r.as / t.r.zs - ((t.r.ms - t.r.mt) + (gp - gq));
-        // H = lse - E[a] = log Z - E[a - m]: ss / zs = E[a], so subtract the maximum first
-        const float ent = gp - (t.ss / t.r.zs - t.r.ms);
+        // H = lse - E[a] = log Z - E[a - m]
+        const float ent = gp - t.ss / t.r.zs;
         if (kl_out) kl_out[n] = kl;
         if (ent_out) ent_out[n] = ent;
         vals[n] = make_float2(kl, ent);

@@ -11,6 +11,9 @@
 
 using namespace fopd;
 
+namespace fopd {
+int host_step_release();  // fopd_host.cu: the host-buffer step's streams and events on the current device
+}
 
 namespace {
 
@@ -19,23 +22,39 @@ std::mutex g_fused_mu;
 
 constexpr int kNotApplicable = 1;  // the on-chip kernel cannot take this shape; use the streaming pair
 
-// Launch shape of the on-chip kernel for one (device, dtype, vocabulary): cluster
-// size, block size, shared memory and how many clusters are resident.
+// Launch shape of the on-chip kernel for one (device, dtype, vocabulary): cluster size, compute
+// warps, vectors per compute thread, shared memory and how many clusters are resident.
 struct FusedPlan {
-  int cluster = 0;     // 0: no shape fits, use the streaming pair
-  int threads = 0;
+  int cluster = 0;        // 0: no shape fits (or the streaming pair is faster), use the streaming pair
+  int nv = 0, warps = 0;  // template parameters: vectors of a slice per compute thread, compute warps
   int slice_vecs = 0;
   size_t smem = 0;
   int max_clusters = 0;
 };
 
 template <int DT>
-const void *fused_kernel_for(int threads) {
-#define X(T) \
-  if (threads == T) return reinterpret_cast<const void *>(&fused_cluster_kernel<DT, T>);
-  FOPD_CLUSTER_THREAD_CHOICES(X)
+const void *fused_kernel_for(int nv, int warps) {
+#define X(N, W) \
+  if (nv == N && warps == W) return reinterpret_cast<const void *>(&fused_cluster_kernel<DT, N, W>);
+  FOPD_FUSED_SHAPES(X)
 #undef X
   return nullptr;
+}
+
+// The instantiated (vectors per thread, compute warps) pair that covers a slice of `slice`
+// vectors with the fewest slots (slots beyond the slice are worked on all the same); among
+// equals the one with more warps.  false: the slice is too long for any.
+static bool fused_shape_for(int64_t slice, int *nv, int *warps) {
+  int64_t best = -1;
+#define X(N, W)                                                                                       \
+  if ((int64_t)N * W * 32 >= slice && (best < 0 || (int64_t)N * W < best || ((int64_t)N * W == best && W > *warps))) { \
+    best = (int64_t)N * W;                                                                             \
+    *nv = N;                                                                                           \
+    *warps = W;                                                                                        \
+  }
+  FOPD_FUSED_SHAPES(X)
+#undef X
+  return best >= 0;
 }
 
 static int set_fused_attributes(const void *kernel, int C, size_t smem) {
@@ -47,14 +66,14 @@ static int set_fused_attributes(const void *kernel, int C, size_t smem) {
   return FOPD_OK;
 }
 
-static void fused_launch_config(cudaLaunchConfig_t *cfg, cudaLaunchAttribute *attr, int C, int threads, size_t smem,
+static void fused_launch_config(cudaLaunchConfig_t *cfg, cudaLaunchAttribute *attr, int C, int warps, size_t smem,
                                 unsigned grid, cudaStream_t st) {
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = C;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
   *cfg = cudaLaunchConfig_t{};
-  cfg->blockDim = dim3(threads);
+  cfg->blockDim = dim3(warps * 32 + 32);
   cfg->gridDim = dim3(grid);
   cfg->dynamicSmemBytes = smem;
   cfg->stream = st;
@@ -62,105 +81,98 @@ static void fused_launch_config(cudaLaunchConfig_t *cfg, cudaLaunchAttribute *at
   cfg->numAttrs = 1;
 }
 
-// Estimated SM cycles a cluster spends on one row: a fixed part per row (barrier hand-offs, the
-// merge of the warps' partial sums, the exchange, which grows with the cluster) plus one round
-// per vector a compute thread sweeps in both sweeps, a round costing in proportion to the warps
-// that share the SM's four schedulers.  Constants fitted to timings on B200 at five vocabularies
-// between 32,000 and 151,936 (blocks of 512-1,024 threads, clusters of 2-12).
-static double row_cycles(int64_t slice, int C, int threads, int ctas_per_sm, double pairs_per_vec) {
-  const int64_t ct = threads - 32, rounds = (slice + ct - 1) / ct;
-  const double per_round = 46.25 * (pairs_per_vec / 8.0) * (double)(threads / 32 - 1) * ctas_per_sm;
-  return 1800.0 + 50.0 * C + (double)rounds * per_round;
+// Shape for one cluster size, or plan->cluster = 0 if that size cannot hold the row: a CTA's
+// slice must be within what its compute threads take (kFusedMaxNV vectors each) and two student
+// and three teacher slices must fit its shared memory.
+template <int DT>
+int fused_plan_for_cluster(int64_t nvec, int C, int max_optin, FusedPlan *plan) {
+  *plan = FusedPlan();
+  const size_t fixed = ((sizeof(ClusterShared) + 127) & ~size_t(127));
+  const int64_t slice = (nvec + C - 1) / C;
+  int nv = 0, warps = 0;
+  const size_t smem = fixed + (size_t)kSliceBufs * (size_t)slice * 16;
+  // (one copy barrier counts < 2^20 bytes)
+  if (!fused_shape_for(slice, &nv, &warps) || smem > (size_t)max_optin || slice * 16 >= (1 << 20)) return FOPD_OK;
+  const void *kernel = fused_kernel_for<DT>(nv, warps);
+  int rc = set_fused_attributes(kernel, C, smem);
+  if (rc != FOPD_OK) return rc;
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[1];
+  fused_launch_config(&cfg, attr, C, warps, smem, (unsigned)C, nullptr);
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) {
+    (void)cudaGetLastError();
+    n = 0;
+  }
+  if (n < 1) return FOPD_OK;
+  plan->cluster = C;
+  plan->nv = nv;
+  plan->warps = warps;
+  plan->slice_vecs = (int)slice;
+  plan->smem = smem;
+  plan->max_clusters = n;
+  return FOPD_OK;
 }
 
-// Picks cluster size and block size with three slice buffers per CTA: the pair with the most
-// rows per cycle = resident clusters (how many clusters of a given size fit depends on how the
-// SMs are grouped) over the estimated cycles per row; among equals the smaller cluster and the
-// larger block.  FOPD_FUSED_CLUSTER / FOPD_FUSED_THREADS in the environment pin them.
+// Picks the cluster size that keeps the most CTAs resident (how many clusters of a given size
+// fit depends on how the SMs are grouped); among equals the smaller cluster (a shorter
+// exchange).  pin > 0: that cluster size or nothing; pin < 0: the streaming pair.
 template <int DT>
-int make_fused_plan(int64_t nvec, FusedPlan *plan) {
+int make_fused_plan(int64_t nvec, int pin, FusedPlan *plan) {
+  *plan = FusedPlan();
+  if (pin < 0) return FOPD_OK;
   int dev = 0, max_optin = 0, n_sm = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&max_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n_sm < 1)
     return FOPD_ERR_CUDA;
-  const size_t fixed = ((sizeof(ClusterShared) + 127) & ~size_t(127));
-  const char *pin_c = getenv("FOPD_FUSED_CLUSTER"), *pin_t = getenv("FOPD_FUSED_THREADS");
-  static const int choices[] = {
-#define X(T) T,
-      FOPD_CLUSTER_THREAD_CHOICES(X)
-#undef X
-  };
   FusedPlan best;
-  double best_score = 0.0;
   for (int C = 1; C <= kMaxClusterSize; ++C) {
-    if (pin_c && atoi(pin_c) != C) continue;
-    const int64_t slice = (nvec + C - 1) / C;
-    const size_t smem = fixed + (size_t)kSliceBufs * 2 * (size_t)slice * 16;
-    if (smem > (size_t)max_optin || slice * 32 >= (1 << 20)) continue;  // one copy barrier counts < 2^20 bytes
-    for (int threads : choices) {
-      if (pin_t && atoi(pin_t) != threads) continue;
-      const void *kernel = fused_kernel_for<DT>(threads);
-      int rc = set_fused_attributes(kernel, C, smem);
-      if (rc != FOPD_OK) return rc;
-      cudaLaunchConfig_t cfg;
-      cudaLaunchAttribute attr[1];
-      fused_launch_config(&cfg, attr, C, threads, smem, (unsigned)C, nullptr);
-      int n = 0;
-      if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess) {
-        (void)cudaGetLastError();
-        n = 0;
-      }
-      if (n < 1) continue;
-      const int ctas_per_sm = (n * C + n_sm - 1) / n_sm;
-      const double score = (double)n / row_cycles(slice, C, threads, ctas_per_sm, Elem<DT>::kPerVec);
-      if (score >= best_score * 1.0001 || (score > best_score * 0.9999 && C == best.cluster)) {
-        best_score = score > best_score ? score : best_score;
-        best.cluster = C;
-        best.threads = threads;
-        best.slice_vecs = (int)slice;
-        best.smem = smem;
-        best.max_clusters = n;
-      }
-    }
+    if (pin > 0 && pin != C) continue;
+    FusedPlan cand;
+    int rc = fused_plan_for_cluster<DT>(nvec, C, max_optin, &cand);
+    if (rc != FOPD_OK) return rc;
+    if (cand.cluster && cand.max_clusters * cand.cluster > best.max_clusters * best.cluster) best = cand;
   }
-  // Against the two streaming sweeps, which move five thirds of the bytes at ~80 % of the
-  // memory system's nominal rate: very long rows leave too few clusters resident for the
-  // on-chip kernel to win, and then the streaming pair is what runs.
-  int sm_khz = 0, mem_khz = 0, bus_bits = 0;
-  if (best.cluster && !pin_c && !pin_t && nvec >= kShortRowVecs &&  // (short rows: both paths are latency-bound)
-      cudaDeviceGetAttribute(&sm_khz, cudaDevAttrClockRate, dev) == cudaSuccess &&
-      cudaDeviceGetAttribute(&mem_khz, cudaDevAttrMemoryClockRate, dev) == cudaSuccess &&
-      cudaDeviceGetAttribute(&bus_bits, cudaDevAttrGlobalMemoryBusWidth, dev) == cudaSuccess && sm_khz > 0 &&
-      mem_khz > 0 && bus_bits > 0) {
-    const double on_chip_s = 1.0 / (best_score * sm_khz * 1e3);
-    const double bytes_per_s = 0.8 * 2.0 * mem_khz * 1e3 * (bus_bits / 8.0);
-    const double pair_s = 5.0 * (double)nvec * 16.0 / bytes_per_s;
-    if (on_chip_s > pair_s) best = FusedPlan();
-  }
+  // The on-chip kernel is bound by instruction issue, so its rate follows the number of resident
+  // CTAs; the two streaming sweeps move five thirds of the bytes at the memory system's rate.
+  // With fewer than about two thirds of the SMs busy (very long rows) the streaming pair wins.
+  if (pin == 0 && best.cluster && best.max_clusters * best.cluster * 3 < n_sm * 2) best = FusedPlan();
   *plan = best;
   return FOPD_OK;
 }
 
+struct PlanEntry {
+  int dev, dtype;
+  int64_t nvec;
+  int pin;      // 0 automatic, > 0 cluster size set by the caller, < 0 streaming pair set by the caller
+  bool planned;
+  FusedPlan plan;
+};
+std::vector<PlanEntry> g_plans;  // guarded by g_fused_mu
+
+// Entry of (current device, dtype, nvec), created on first use.  Caller holds g_fused_mu.
+PlanEntry *plan_entry(int dtype, int64_t nvec) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+  for (PlanEntry &e : g_plans)
+    if (e.dev == dev && e.dtype == dtype && e.nvec == nvec) return &e;
+  g_plans.push_back({dev, dtype, nvec, 0, false, FusedPlan()});
+  return &g_plans.back();
+}
+
 template <int DT>
 int fused_plan(int64_t nvec, FusedPlan *plan) {
-  struct Entry {
-    int dev;
-    int64_t nvec;
-    FusedPlan plan;
-  };
-  static std::vector<Entry> cache;
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return FOPD_ERR_CUDA;
   std::lock_guard<std::mutex> lock(g_fused_mu);
-  for (const Entry &e : cache)
-    if (e.dev == dev && e.nvec == nvec) {
-      *plan = e.plan;
-      return FOPD_OK;
-    }
-  int rc = make_fused_plan<DT>(nvec, plan);
-  if (rc == FOPD_OK) cache.push_back({dev, nvec, *plan});
-  return rc;
+  PlanEntry *e = plan_entry(DT, nvec);
+  if (!e) return FOPD_ERR_CUDA;
+  if (!e->planned) {
+    int rc = make_fused_plan<DT>(nvec, e->pin, &e->plan);
+    if (rc != FOPD_OK) return rc;
+    e->planned = true;
+  }
+  *plan = e->plan;
+  return FOPD_OK;
 }
 
 // Fused on-chip forward + backward (cluster_kernel.cuh).  tmp holds [n_rows, 4] row
@@ -176,7 +188,7 @@ int launch_fused(const fopd_chunk *chunk, int32_t B, const float *coef, float la
   if (rc != FOPD_OK) return rc;
   if (!plan.cluster || plan.max_clusters < 1) return kNotApplicable;
   const int C = plan.cluster;
-  const void *kernel = fused_kernel_for<DT>(plan.threads);
+  const void *kernel = fused_kernel_for<DT>(plan.nv, plan.warps);
   float *row_cf = tmp + 4 * chunk->n_rows;
   const ChunkDev d = to_dev(chunk);
   row_coef_kernel<<<(unsigned)((chunk->n_rows + 255) / 256), 256, 0, st>>>(d, B, coef, status, row_cf);
@@ -184,7 +196,7 @@ int launch_fused(const fopd_chunk *chunk, int32_t B, const float *coef, float la
   const int64_t clusters = chunk->n_rows < plan.max_clusters ? chunk->n_rows : plan.max_clusters;
   cudaLaunchConfig_t cfg;
   cudaLaunchAttribute attr[1];
-  fused_launch_config(&cfg, attr, C, plan.threads, plan.smem, (unsigned)(clusters * C), st);
+  fused_launch_config(&cfg, attr, C, plan.warps, plan.smem, (unsigned)(clusters * C), st);
   FusedArgs a;
   a.c = d;
   a.lambda = lambda;
@@ -193,6 +205,7 @@ int launch_fused(const fopd_chunk *chunk, int32_t B, const float *coef, float la
   a.row_ws = tmp;
   a.status = status;
   a.slice_vecs = plan.slice_vecs;
+  a.wait_cycles = kWaitCycles;
   void *args[] = {&a};
   // the attributes are per function, and the plan of another vocabulary may have changed them:
   // set them and launch under one lock, so that a call from another thread cannot come between
@@ -326,10 +339,43 @@ int fopd_loss_fwd_bwd_plan(int32_t dtype, int64_t vocab, int32_t *cluster_size, 
   if (nvec >= 1) rc = dtype == FOPD_BF16 ? fused_plan<FOPD_BF16>(nvec, &plan) : fused_plan<FOPD_F32>(nvec, &plan);
   if (rc != FOPD_OK) return rc;
   if (cluster_size) *cluster_size = plan.cluster;
-  if (block_threads) *block_threads = plan.threads;
+  if (block_threads) *block_threads = plan.cluster ? plan.warps * 32 + 32 : 0;
   if (resident_clusters) *resident_clusters = plan.max_clusters;
   if (smem_bytes) *smem_bytes = (int32_t)plan.smem;
   return FOPD_OK;
+}
+
+int fopd_loss_fwd_bwd_set_plan(int32_t dtype, int64_t vocab, int32_t cluster_size) {
+  if (dtype != FOPD_BF16 && dtype != FOPD_F32) return FOPD_ERR_DTYPE;
+  if (vocab <= 0 || vocab > (int64_t)1 << 30 || cluster_size > kMaxClusterSize) return FOPD_ERR_SIZE;
+  const int64_t nvec = vocab / (dtype == FOPD_BF16 ? 8 : 4);
+  if (nvec < 1) return cluster_size > 0 ? FOPD_ERR_SIZE : FOPD_OK;
+  const int pin = cluster_size < 0 ? -1 : cluster_size;
+  FusedPlan plan;
+  std::lock_guard<std::mutex> lock(g_fused_mu);
+  int rc = dtype == FOPD_BF16 ? make_fused_plan<FOPD_BF16>(nvec, pin, &plan) : make_fused_plan<FOPD_F32>(nvec, pin, &plan);
+  if (rc != FOPD_OK) return rc;
+  if (pin > 0 && !plan.cluster) return FOPD_ERR_SIZE;  // that cluster size cannot hold the row on this device
+  PlanEntry *e = plan_entry(dtype, nvec);
+  if (!e) return FOPD_ERR_CUDA;
+  e->pin = pin;
+  e->plan = plan;
+  e->planned = true;
+  return FOPD_OK;
+}
+
+int fopd_selftest_bounded_wait(int64_t limit_cycles, int32_t *status, int64_t *waited_cycles, void *stream) {
+  if (!status) return FOPD_ERR_NULL;
+  if (limit_cycles < 0 || limit_cycles > kWaitCycles) return FOPD_ERR_SIZE;
+  bounded_wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(
+      (long long)limit_cycles, status, reinterpret_cast<long long *>(waited_cycles));
+  return launch_ok();
+}
+
+int fopd_release_device_memory(void) {
+  int rc = scratch_release();
+  const int rc2 = host_step_release();
+  return rc != FOPD_OK ? rc : rc2;
 }
 
 int fopd_loss_finalize(const double *loss_acc, const double *acc, const float *w, int32_t B,

@@ -150,6 +150,31 @@ int get_pipe(Pipe **out) {
   return FOPD_OK;
 }
 
+}  // namespace
+
+namespace fopd {
+// Destroys the current device's streams and events of the pipelined path (they are made again
+// on the next host-buffer step).  Waits for a step in progress on that device.
+int host_step_release() {
+  int d = 0;
+  if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= 64) return FOPD_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_pipe_mu[d]);
+  Pipe &P = g_pipes[d];
+  if (!P.ok) return FOPD_OK;
+  bool fine = cudaStreamDestroy(P.compute) == cudaSuccess;
+  fine = (cudaStreamDestroy(P.down) == cudaSuccess) && fine;
+  fine = (cudaEventDestroy(P.up) == cudaSuccess) && fine;
+  fine = (cudaEventDestroy(P.grad) == cudaSuccess) && fine;
+  fine = (cudaEventDestroy(P.fin) == cudaSuccess) && fine;
+  for (int k = 0; k < kMaxSlots; ++k) fine = (cudaEventDestroy(P.slot_free[k]) == cudaSuccess) && fine;
+  P = Pipe();
+  if (!fine) (void)cudaGetLastError();
+  return fine ? FOPD_OK : FOPD_ERR_CUDA;
+}
+}  // namespace fopd
+
+namespace {
+
 // rows [a, b) of a chunk as a chunk of its own
 fopd_chunk sub_chunk(const fopd_chunk &c, int64_t a, int64_t b) {
   fopd_chunk s = c;

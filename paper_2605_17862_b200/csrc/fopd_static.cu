@@ -15,7 +15,6 @@ static __device__ __align__(256) float g_static_row_ws[(size_t)FOPD_STATIC_MAX_R
 
 namespace {
 
-constexpr int kMaxDevices = 64;
 std::mutex g_setup_mutex;
 float *g_static_row_ws_addr[kMaxDevices] = {};
 
@@ -27,8 +26,10 @@ int static_scratch(float **out) {
   std::lock_guard<std::mutex> lock(g_setup_mutex);
   if (!g_static_row_ws_addr[dev]) {
     float *ptr = nullptr;
-    if (cudaGetSymbolAddress(reinterpret_cast<void **>(&ptr), g_static_row_ws) != cudaSuccess || !ptr)
+    if (cudaGetSymbolAddress(reinterpret_cast<void **>(&ptr), g_static_row_ws) != cudaSuccess || !ptr) {
+      (void)cudaGetLastError();  // leave no sticky-looking error behind for the caller's next check
       return FOPD_ERR_CUDA;
+    }
     g_static_row_ws_addr[dev] = ptr;
   }
   *out = g_static_row_ws_addr[dev];

@@ -52,16 +52,24 @@ static inline int launch_ok() { return cudaGetLastError() == cudaSuccess ? FOPD_
 // that keeps what it has been given: with the device's default pool a synchronisation
 // between two calls hands the memory back to the driver and the next call pays for a
 // fresh allocation, which costs more than the kernels.
+constexpr int kMaxDevices = 64;
+struct ScratchPools {
+  std::mutex mu;
+  cudaMemPool_t pools[kMaxDevices] = {};
+};
+inline ScratchPools &scratch_pools() {
+  static ScratchPools p;  // one per process (inline function: one instance across translation units)
+  return p;
+}
+
 static inline int scratch_alloc(void **ptr, size_t bytes, cudaStream_t st) {
-  constexpr int kMaxDevices = 64;
-  static std::mutex mu;
-  static cudaMemPool_t pools[kMaxDevices] = {};
+  ScratchPools &sp = scratch_pools();
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return FOPD_ERR_CUDA;
   cudaMemPool_t pool;
   {
-    std::lock_guard<std::mutex> lock(mu);
-    if (!pools[dev]) {
+    std::lock_guard<std::mutex> lock(sp.mu);
+    if (!sp.pools[dev]) {
       cudaMemPoolProps props = {};
       props.allocType = cudaMemAllocationTypePinned;
       props.location.type = cudaMemLocationTypeDevice;
@@ -73,11 +81,21 @@ static inline int scratch_alloc(void **ptr, size_t bytes, cudaStream_t st) {
         (void)cudaMemPoolDestroy(created);
         return FOPD_ERR_CUDA;
       }
-      pools[dev] = created;
+      sp.pools[dev] = created;
     }
-    pool = pools[dev];
+    pool = sp.pools[dev];
   }
   return cudaMallocFromPoolAsync(ptr, bytes, pool, st) == cudaSuccess ? FOPD_OK : FOPD_ERR_CUDA;
+}
+
+// Gives the memory the current device's pool holds but no pending call uses back to the driver.
+static inline int scratch_release() {
+  ScratchPools &sp = scratch_pools();
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return FOPD_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(sp.mu);
+  if (!sp.pools[dev]) return FOPD_OK;
+  return cudaMemPoolTrimTo(sp.pools[dev], 0) == cudaSuccess ? FOPD_OK : FOPD_ERR_CUDA;
 }
 
 // One CTA per row.

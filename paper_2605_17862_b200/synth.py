@@ -56,7 +56,14 @@ class Workload:
 # prints values for alpha, beta, xi, lambda (they are tuned on a pilot split),
 # so these are this repository's choice: with xi = 0.15 a sample with
 # staleness >= 6 is always gated out and staleness 4-5 sits near the gate.
-DEFAULT_PARAMS = dict(alpha=1.0, beta=1.0, xi=0.15, lam=0.1)
+def f32_params(alpha=1.0, beta=1.0, xi=0.15, lam=0.1) -> dict:
+    """Hyper-parameters rounded to fp32 once, as Python floats.  The C ABI carries
+    them as ``float``; a checker that is to see identical inputs must be handed
+    these rounded values, not the decimal literals (0.15 is not an fp32 number)."""
+    return {k: float(np.float32(v)) for k, v in dict(alpha=alpha, beta=beta, xi=xi, lam=lam).items()}
+
+
+DEFAULT_PARAMS = f32_params()
 
 
 def _scaled_vocab(full: int, scale: float) -> int:

@@ -21,7 +21,15 @@ from paper_2605_17862_b200 import pipeline as pl
 TOL_LOGPROB = 1e-3
 TOL_REL = 1e-4
 TOL_GRAD_ABS = 1e-5
-PARAMS = dict(alpha=1.0, beta=1.0, xi=0.15, lam=0.1)
+from paper_2605_17862_b200 import synth
+
+# The library takes alpha, beta, xi, lambda as C floats: both sides get the fp32-rounded values.
+PARAMS = synth.f32_params()
+
+
+def exact(params):
+    """Any parameter dict (e.g. ``dict(PARAMS, xi=0.05)``) rounded to fp32 for both sides."""
+    return synth.f32_params(**params)
 
 
 def host_chunk(d):
@@ -30,6 +38,7 @@ def host_chunk(d):
 
 def gpu_run(chunks_dev, B, tau, H, d_sup=None, params=PARAMS, use_row_ws=True, vocab=None, want_rows=True):
     dev = chunks_dev[0]["student"].device
+    params = exact(params)
     chunks = [pl.to_chunk(c, vocab) for c in chunks_dev]
     buf = pl.BatchBuffers(B, dev)
     rows = [pl.RowOutputs.alloc(c["student"].shape[0], dev) for c in chunks_dev]
@@ -45,6 +54,7 @@ def gpu_run(chunks_dev, B, tau, H, d_sup=None, params=PARAMS, use_row_ws=True, v
 
 
 def oracle_run(chunks_host, B, tau, H, d_sup=None, params=PARAMS):
+    params = exact(params)
     return orc.run_batch(chunks_host, B, tau, H, d_sup, params["alpha"], params["beta"], params["xi"], params["lam"])
 
 
@@ -63,6 +73,7 @@ def gpu_run_vocab_sharded(cuts):
         dev = chunks_dev[0]["student"].device
         V = vocab or chunks_dev[0]["student"].shape[1]
         assert cuts[0] == 0 and cuts[-1] == V
+        params = exact(params)
         p = fb.params(**params)
         tau_d = torch.as_tensor(np.asarray(tau, dtype=np.int32), device=dev)
         H_d = torch.as_tensor(np.asarray(H, dtype=np.int32), device=dev)
@@ -109,6 +120,7 @@ def gpu_run_vocab_sharded(cuts):
 def compare(chunks_dev, B, tau, H, d_sup=None, params=PARAMS, use_row_ws=True, grad_rows_per_chunk=None,
             seed=0, expect_bits=0, vocab=None, runner=None):
     """Full comparison of one batch; returns a dict of the maxima seen."""
+    params = exact(params)
     buf, rows, dlogits, bits = (runner or gpu_run)(chunks_dev, B, tau, H, d_sup, params, use_row_ws, vocab)
     assert bits == expect_bits, f"device status bits {bits}"
     V = vocab or chunks_dev[0]["student"].shape[1]
@@ -218,6 +230,7 @@ def compare(chunks_dev, B, tau, H, d_sup=None, params=PARAMS, use_row_ws=True, g
         # of the difference belongs to the weight, not to the gradient sweep
         cf_gpu = buf.coef.cpu().numpy().astype(np.float64)
         rel_w = np.where(fr.coef > 0, np.abs(cf_gpu - fr.coef) / np.maximum(fr.coef, 1e-300), 0.0)
+        out["w_rel"] = max(out.get("w_rel", 0.0), float(rel_w.max()))
         bound += rel_w[np.clip(c["sample_id"].numpy()[sel], 0, B - 1)][:, None] * np.abs(g_ref)
         ycol = np.clip(c["tokens"].numpy()[sel], 0, V - 1)
         # d = lp_s - b carries the absolute fp32 error of the log-normaliser (~1e-6), so the

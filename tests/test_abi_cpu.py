@@ -31,7 +31,7 @@ def test_library_exports_every_declared_symbol(lib):
     for n in names:
         assert hasattr(lib, n), f"{n} declared in fopd.h but not exported"
     assert set(names) == set(fb.EXPORTS)
-    assert fb.version() == 100
+    assert fb.version() == 200
 
 
 def test_strerror_covers_every_status(lib):
@@ -139,3 +139,14 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(fb, "LIB_PATH", str(tmp_path / "libfopd.so"))
     with pytest.raises(FileNotFoundError):
         fb.lib()
+
+
+def test_new_control_entry_points_check_their_arguments_on_the_host(lib):
+    """No GPU: these return before any CUDA call."""
+    assert lib.fopd_loss_fwd_bwd_set_plan(7, 151936, 4) == -4          # dtype
+    assert lib.fopd_loss_fwd_bwd_set_plan(0, 0, 4) == -3               # vocabulary
+    assert lib.fopd_loss_fwd_bwd_set_plan(0, 151936, 17) == -3         # more CTAs than a cluster can have
+    assert lib.fopd_selftest_bounded_wait(1000, None, None, None) == -1
+    status = ctypes.c_void_p(0x1000)
+    assert lib.fopd_selftest_bounded_wait(-1, status, None, None) == -3
+    assert lib.fopd_selftest_bounded_wait(10**12, status, None, None) == -3

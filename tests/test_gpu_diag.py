@@ -109,6 +109,26 @@ def test_row_divergence_shapes_entropy_and_student_teacher_kl(V, stride, dtype):
     assert bits == 2 and k_b[-1] == 0.0
 
 
+@pytest.mark.parametrize("offset,dtype", [(200.0, torch.bfloat16), (-300.0, torch.bfloat16), (100.0, torch.float32),
+                                          (-1000.0, torch.float32)])
+def test_row_divergence_with_large_logit_offsets(offset, dtype):
+    """KL and entropy are shift invariant: logits far from zero (both tensors shifted, and the
+    second shifted by a further 50) must give the oracle's values on the same shifted bits."""
+    wl = synth.tiny(scale=1 / 8) if dtype == torch.float32 else synth.reasoning(scale=1 / 32)
+    ch = synth.gen_chunk(wl, 0, DEV)
+    first = (ch["student"].float() + offset).to(dtype)
+    second = (ch["teacher"].float() + offset + 50.0).to(dtype)
+    lo, hi = wl.chunk_range(0)
+    mask = wl.mask[lo:hi]
+    k_g, e_g, acc, bits = _divergence(first, second, ch["mask"], ch["sample_id"], wl.B)
+    k_o, e_o = orc.row_divergence(first.cpu(), second.cpu(), mask)
+    mb = mask.astype(bool)
+    assert bits == 0 and mb.any()
+    assert np.abs(k_g - k_o)[mb].max() <= 1e-4 * max(1.0, k_o.max())
+    assert np.abs(e_g - e_o)[mb].max() <= 1e-4 * max(1.0, e_o.max())
+    print(offset, np.abs(k_g - k_o)[mb].max(), np.abs(e_g - e_o)[mb].max())
+
+
 def test_refresh_decision_against_oracle():
     rng = np.random.default_rng(3)
     cases = []

@@ -23,6 +23,7 @@ def _host_chunks(wl, row_stride=None):
 
 
 def _run_host(host, B, tau, H, d_sup, params, resident, vocab=None):
+    params = par.exact(params)
     hchunks = [pl.to_chunk(c, vocab) for c in host]
     need = fb.fopd_step_host_workspace_bytes(hchunks, B, resident)
     assert need > 0
@@ -38,6 +39,7 @@ def _run_host(host, B, tau, H, d_sup, params, resident, vocab=None):
 
 
 def _check(host, B, tau, H, d_sup=None, params=par.PARAMS, resident=True, vocab=None, expect_bits=0):
+    params = par.exact(params)
     res, dl = _run_host(host, B, tau, H, d_sup, params, resident, vocab)
     assert int(res["status_bits"][0]) == expect_bits
     V = vocab or host[0]["student"].shape[1]
