@@ -23,7 +23,15 @@
  *     loss path uses one set for both;
  *   - the gate w_i = ReLU(f_i - xi) is a constant in the backward pass;
  *   - the batch mean of Eq. 16 / Algorithm 1 divides by the number of samples
- *     passed in, gated and invalid ones included.
+ *     passed in, gated and invalid ones included;
+ *   - the sampled-token form of the token loss (the setup Sec. 5 says the
+ *     experiments follow, and the sampled-token objectives of Appendix B) is
+ *     rho_n (log p_s(y_n) - log p_t(y_n)) on the stored token y_n ~ pi^r, with
+ *     rho_n = pi^t(y_n) / pi^r(y_n): its expectation under pi^r is the
+ *     full-vocabulary reverse KL of Eq. 12.  In its gradient the importance
+ *     ratio carries the derivative and the log-ratio is a constant (the reward
+ *     of a policy-gradient step), whose expectation under pi^r is the gradient
+ *     of that KL.
  *
  * Pins (tests/test_oracle_pins.py): every function here is pinned to closed
  * forms, brute force on tiny vocabularies, library routines in float64,
@@ -282,6 +290,69 @@ void oracle_grad_rows(const void *student, const void *teacher, int dtype,
             double p = exp(logp);
             double onehot = (v == tokens[n]) ? 1.0 : 0.0;
             g[v] = c * (p * ((logp - logq) - kln) + lambda * rho_d * (onehot - p));
+        }
+    }
+}
+
+/*
+ * Sampled-token form of the token loss of Eq. 12 (Sec. 5, experimental setup;
+ * Appendix B, sampled-token objectives): for an aligned row n with stored token
+ * y_n ~ pi^r and rho_n = pi^t(y_n) / pi^r(y_n),
+ *
+ *   l_n = rho_n ( log p_s(y_n) - log p_t(y_n) )
+ *
+ * whose expectation over y ~ pi^r is sum_y p_s(y) (log p_s(y) - log p_t(y)).
+ * out[n] = l_n for aligned rows, 0 otherwise.  lp_s, lp_t, rho, valid are the
+ * arrays oracle_token_stats wrote.
+ */
+void oracle_sampled_token_loss(int64_t n_rows, const double *lp_s, const double *lp_t,
+                               const double *rho, const uint8_t *valid, double *out) {
+    for (int64_t n = 0; n < n_rows; ++n)
+        out[n] = valid[n] ? rho[n] * (lp_s[n] - lp_t[n]) : 0.0;
+}
+
+/*
+ * Gradient with respect to the student logits of selected rows for the
+ * sampled-token loss, with w_i and the log-ratio r_n = log p_s(y_n) - log p_t(y_n)
+ * held constant and the importance ratio rho_n = exp(log p_s(y_n) - b_n)
+ * differentiated (d rho_n / dS_v = rho_n (1[v = y_n] - p_s(v))); the rollout
+ * anchor lambda * k3(rho_n) as in oracle_grad_rows.  For c = coef_i:
+ *
+ *   dS[n, v] = c ( rho_n r_n + lambda rho_n d_n ) ( 1[v = y_n] - p_s(v) )
+ *
+ * Rows that are not aligned, or whose sample has coef = 0, get zeros.
+ */
+void oracle_grad_rows_sampled(const void *student, const void *teacher, int dtype,
+                              int64_t V, int64_t row_stride, const int32_t *tokens,
+                              const float *behav_logprob, const uint8_t *mask,
+                              const int32_t *sample_id, int32_t B, const double *coef,
+                              double lambda, const int64_t *rows, int64_t n_sel,
+                              double *out) {
+    size_t esz = dtype == ORACLE_BF16 ? 2 : 4;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t k = 0; k < n_sel; ++k) {
+        int64_t n = rows[k];
+        double *g = out + (size_t)k * V;
+        int ok = mask[n] != 0 && tokens[n] >= 0 && tokens[n] < V &&
+                 sample_id[n] >= 0 && sample_id[n] < B;
+        double c = ok ? coef[sample_id[n]] : 0.0;
+        if (c == 0.0) {
+            for (int64_t v = 0; v < V; ++v) g[v] = 0.0;
+            continue;
+        }
+        const void *srow = (const char *)student + (size_t)n * row_stride * esz;
+        const void *trow = (const char *)teacher + (size_t)n * row_stride * esz;
+        double ls = row_logsumexp(srow, dtype, V);
+        double lt = row_logsumexp(trow, dtype, V);
+        double lps = logit_at(srow, dtype, tokens[n]) - ls;
+        double lpt = logit_at(trow, dtype, tokens[n]) - lt;
+        double dn = lps - (double)behav_logprob[n];
+        double rho = exp(dn);
+        double weight = c * (rho * (lps - lpt) + lambda * rho * dn);
+        for (int64_t v = 0; v < V; ++v) {
+            double p = exp(logit_at(srow, dtype, v) - ls);
+            double onehot = (v == tokens[n]) ? 1.0 : 0.0;
+            g[v] = weight * (onehot - p);
         }
     }
 }

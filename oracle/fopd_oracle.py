@@ -165,7 +165,21 @@ def loss(fr: Freshness, lam):
     return float(total), per
 
 
-def grad_rows(student, teacher, tokens, behav_logprob, mask, sample_id, coef, lam, rows):
+FULL_KL, SAMPLED_KL = 0, 1  # forms of the token loss of Eq. 12
+
+
+def token_loss(st: TokenStats, loss_kind: int = FULL_KL) -> np.ndarray:
+    """Per-token loss of a chunk: the full-vocabulary reverse KL (loss_kind 0) or its
+    sampled-token form rho_n (lp_s - lp_t) on the stored token (loss_kind 1)."""
+    if loss_kind == FULL_KL:
+        return st.kl
+    out = np.zeros_like(st.kl)
+    lib().oracle_sampled_token_loss(ctypes.c_int64(len(out)), _p(st.lp_s), _p(st.lp_t), _p(st.rho),
+                                    _p(st.valid), _p(out))
+    return out
+
+
+def grad_rows(student, teacher, tokens, behav_logprob, mask, sample_id, coef, lam, rows, loss_kind: int = FULL_KL):
     """d L / d student logits for the listed rows, [len(rows), V] float64."""
     S, dt = _logits(student)
     T, dt2 = _logits(teacher)
@@ -179,7 +193,8 @@ def grad_rows(student, teacher, tokens, behav_logprob, mask, sample_id, coef, la
     rows = _np(rows, np.int64)
     assert rows.size == 0 or (rows.min() >= 0 and rows.max() < n)
     out = np.zeros((len(rows), V), dtype=np.float64)
-    lib().oracle_grad_rows(
+    fn = lib().oracle_grad_rows if loss_kind == FULL_KL else lib().oracle_grad_rows_sampled
+    fn(
         _p(S), _p(T), ctypes.c_int(dt), ctypes.c_int64(V), ctypes.c_int64(V), _p(y), _p(b), _p(mk),
         _p(sid), ctypes.c_int32(len(coef)), _p(coef), ctypes.c_double(lam), _p(rows),
         ctypes.c_int64(len(rows)), _p(out),
@@ -298,7 +313,7 @@ class BatchResult:
     per_sample_loss: np.ndarray
 
 
-def run_batch(chunks, B, tau, H, d_sup, alpha, beta, xi, lam) -> BatchResult:
+def run_batch(chunks, B, tau, H, d_sup, alpha, beta, xi, lam, loss_kind: int = FULL_KL) -> BatchResult:
     """Algorithm 1's measurement phase then its minibatch objective, over a
     batch supplied as a list of chunks.  Each chunk is a dict with keys
     student, teacher, tokens, behav_logprob, mask, sample_id."""
@@ -307,6 +322,8 @@ def run_batch(chunks, B, tau, H, d_sup, alpha, beta, xi, lam) -> BatchResult:
     for c in chunks:
         st = token_stats(c["student"], c["teacher"], c["tokens"], c["behav_logprob"],
                          c["mask"], c["sample_id"], B)
+        if loss_kind != FULL_KL:  # the per-sample mean of Eq. 12 is taken over this form of the token loss
+            st.kl = token_loss(st, loss_kind)
         sample_accumulate(acc, c["sample_id"], st)
         stats.append(st)
     fr = sample_freshness(acc, tau, H, d_sup, alpha, beta, xi)

@@ -539,3 +539,116 @@ def test_merged_shard_partials_equal_whole_row_statistics(dtype):
     # a token outside every part is reported as not found
     far = orc.shard_partials(S[:, :10].contiguous(), T[:, :10].contiguous(), np.full(n, 200, np.int32), mask, 0)
     assert np.all(orc.merge_partials([far])[5] == 0)
+
+
+# ------------------------------------------------- sampled-token form of the token loss
+def test_sampled_token_loss_expectation_is_the_full_vocabulary_reverse_kl():
+    # Enumerate every y on a tiny vocabulary, y ~ pi_r:
+    #   sum_y pi_r(y) rho(y) (log p_s(y) - log p_t(y)) = KL(p_s || p_t)        (Eq. 12)
+    # with rho(y) = p_s(y) / pi_r(y); exact when pi_r is carried as the fp32 log-probs the path gets.
+    rng = np.random.default_rng(31)
+    for V in (2, 5, 13):
+        s = (rng.standard_normal(V) * 1.5).astype(np.float32)
+        t = (s + rng.standard_normal(V)).astype(np.float32)
+        old = s + rng.standard_normal(V) * 0.7
+        b = torch.log_softmax(torch.tensor(old, dtype=torch.float64), 0).numpy().astype(np.float32)
+        S, T = np.tile(s, (V, 1)), np.tile(t, (V, 1))
+        st = _stats(S, T, np.arange(V, dtype=np.int32), b)
+        tl = orc.token_loss(st, orc.SAMPLED_KL)
+        pr = np.exp(b.astype(np.float64))
+        lhs = float(np.sum(pr * tl))
+        assert abs(lhs - st.kl[0]) < 1e-12          # the oracle's own full-vocabulary token loss
+        lp_s = torch.log_softmax(torch.tensor(s, dtype=torch.float64), 0)
+        lp_t = torch.log_softmax(torch.tensor(t, dtype=torch.float64), 0)
+        assert abs(lhs - float(torch.sum(lp_s.exp() * (lp_s - lp_t)))) < 1e-12   # and the definition
+        # the other direction of the KL is a different number
+        assert abs(lhs - float(torch.sum(lp_t.exp() * (lp_t - lp_s)))) > 1e-3
+        # a single sampled term may be negative, the full-vocabulary loss is not
+        assert tl.min() < 0 < st.kl[0]
+
+
+def test_sampled_token_loss_special_cases():
+    rng = np.random.default_rng(32)
+    S, T, y, _ = _rand_rows(rng, 6, 9)
+    lp = torch.log_softmax(torch.from_numpy(S).double(), 1).numpy()[np.arange(6), y]
+    # behaviour = current and teacher = student: ratio 1, log-ratio 0, loss 0, gradient 0
+    st = _stats(S, S, y, lp.astype(np.float32))
+    assert np.all(orc.token_loss(st, orc.SAMPLED_KL) == 0.0)
+    coef = np.array([0.25])
+    g = orc.grad_rows(S, S, y, lp.astype(np.float32), np.ones(6, np.uint8), np.zeros(6, np.int32), coef, 0.3,
+                      np.arange(6), loss_kind=orc.SAMPLED_KL)
+    assert np.abs(g).max() < 1e-7   # d = lp_s - fp32(lp_s) is a rounding residue, not zero
+    # hand value: V = 2, s = (0, ln 3), t = (0, 0), token 1, behaviour log-prob ln(1/2):
+    # p_s = (1/4, 3/4), p_t = (1/2, 1/2), rho = (3/4)/(1/2) = 3/2, r = ln(3/2), loss = 1.5 ln 1.5
+    s2 = np.array([[0.0, math.log(3.0)]], np.float32)
+    t2 = np.zeros((1, 2), np.float32)
+    st2 = _stats(s2, t2, np.array([1], np.int32), np.array([math.log(0.5)], np.float32))
+    assert abs(orc.token_loss(st2, orc.SAMPLED_KL)[0] - 1.5 * math.log(1.5)) < 1e-6
+    # masked rows contribute nothing
+    m = np.array([1, 0, 1, 1, 0, 1], np.uint8)
+    stm = _stats(S, T, y, lp.astype(np.float32), mask=m)
+    tlm = orc.token_loss(stm, orc.SAMPLED_KL)
+    assert np.all(tlm[m == 0] == 0.0) and np.all(tlm[m == 1] != 0.0)
+
+
+def test_sampled_gradient_expectation_is_the_full_vocabulary_gradient():
+    # sum_y pi_r(y) * (gradient of the sampled form with token y) = gradient of the full-vocabulary
+    # form, for lambda = 0 (the anchor is the same term in both forms and is pinned separately)
+    rng = np.random.default_rng(33)
+    for V in (3, 7):
+        s = (rng.standard_normal(V) * 1.5).astype(np.float32)
+        t = (s + rng.standard_normal(V)).astype(np.float32)
+        b = torch.log_softmax(torch.tensor(s + rng.standard_normal(V) * 0.5, dtype=torch.float64), 0).numpy().astype(np.float32)
+        S, T = np.tile(s, (V, 1)), np.tile(t, (V, 1))
+        y = np.arange(V, dtype=np.int32)
+        ones, zeros = np.ones(V, np.uint8), np.zeros(V, np.int32)
+        coef = np.array([1.0])
+        gs = orc.grad_rows(S, T, y, b, ones, zeros, coef, 0.0, np.arange(V), loss_kind=orc.SAMPLED_KL)
+        gf = orc.grad_rows(S, T, y, b, ones, zeros, coef, 0.0, np.array([0]))
+        pr = np.exp(b.astype(np.float64))[:, None]
+        assert np.abs((pr * gs).sum(0) - gf[0]).max() < 1e-12
+
+
+def test_sampled_gradient_matches_central_finite_differences_and_structure():
+    rng = np.random.default_rng(34)
+    chunk, tau, H = _tiny_batch(rng, V=7)
+    B, lam = 3, 0.37
+    r = orc.run_batch([chunk], B, tau, H, None, 1.0, 1.0, 0.05, lam, loss_kind=orc.SAMPLED_KL)
+    assert np.all(r.fresh.w > 0)
+    n, V = chunk["student"].shape
+    g = orc.grad_rows(chunk["student"], chunk["teacher"], chunk["tokens"], chunk["behav_logprob"],
+                      chunk["mask"], chunk["sample_id"], r.fresh.coef, lam, np.arange(n), loss_kind=orc.SAMPLED_KL)
+    st0 = r.stats[0]
+    reward = st0.lp_s - st0.lp_t          # held constant: the importance ratio carries the derivative
+    cnt = np.bincount(chunk["sample_id"][st0.valid.astype(bool)], minlength=B)
+
+    def surrogate(S):
+        st = orc.token_stats(S, chunk["teacher"], chunk["tokens"], chunk["behav_logprob"], chunk["mask"],
+                             chunk["sample_id"], B)
+        per_tok = st.valid * (st.rho * reward + lam * st.k3)
+        tot = 0.0
+        for i in range(B):
+            tot += r.fresh.w[i] * per_tok[chunk["sample_id"] == i].sum() / cnt[i]
+        return tot / B
+
+    h = np.float32(2.0 ** -9)
+    fd = np.zeros((n, V))
+    for i in range(n):
+        for v in range(V):
+            Sp, Sm = chunk["student"].copy(), chunk["student"].copy()
+            Sp[i, v] += h
+            Sm[i, v] -= h
+            fd[i, v] = (surrogate(Sp) - surrogate(Sm)) / (float(Sp[i, v]) - float(Sm[i, v]))
+    assert np.all(g[1] == 0.0) and np.all(fd[1] == 0.0)   # masked row
+    assert np.max(np.abs(g - fd)) < 2e-5 * np.abs(g).max()
+    assert np.abs(g.sum(1)).max() < 1e-15                  # tangent to the simplex
+    # the per-sample loss is the mean of the sampled token losses, the objective as in Eq. 16
+    tl = orc.token_loss(orc.token_stats(chunk["student"], chunk["teacher"], chunk["tokens"], chunk["behav_logprob"],
+                                        chunk["mask"], chunk["sample_id"], B), orc.SAMPLED_KL)
+    ell = np.array([tl[(chunk["sample_id"] == i) & (chunk["mask"] == 1)].mean() for i in range(B)])
+    assert np.allclose(r.fresh.ell, ell, rtol=1e-14)
+    assert abs(r.loss - float(np.mean(r.fresh.w * (ell + lam * r.fresh.D_roll)))) < 1e-15
+    # a gated sample's rows get zeros
+    gated = orc.grad_rows(chunk["student"], chunk["teacher"], chunk["tokens"], chunk["behav_logprob"], chunk["mask"],
+                          chunk["sample_id"], np.array([0.1, 0.0, 0.2]), lam, np.arange(n), loss_kind=orc.SAMPLED_KL)
+    assert np.all(gated[chunk["sample_id"] == 1] == 0.0)
