@@ -77,6 +77,24 @@ extern "C" {
 
 typedef enum { FOPD_BF16 = 0, FOPD_F32 = 1 } fopd_dtype;
 
+/*
+ * Form of the token loss l(pi_theta, pi_teacher) of Eq. 12, which the paper leaves generic.
+ *
+ *   FOPD_LOSS_FULL_KL     kl_n = sum_v p_s(v) (log p_s(v) - log p_t(v)), the reverse KL over the
+ *                         whole vocabulary (the default everywhere in this header).
+ *   FOPD_LOSS_SAMPLED_KL  l_n = rho_n (log p_s(y_n) - log p_t(y_n)) on the stored token y_n,
+ *                         rho_n = pi^t(y_n) / pi^r(y_n): the sampled-token reverse KL with an
+ *                         importance ratio of the setup Sec. 5 says the experiments follow
+ *                         (Appendix B's sampled-token objectives).  Its expectation over y_n
+ *                         drawn from the behaviour policy is kl_n.  In the gradient the ratio
+ *                         carries the derivative and the log-ratio is a constant (the reward of
+ *                         a policy-gradient step):
+ *                           dlogits[n,v] = coef_i rho_n ( (log p_s(y_n) - log p_t(y_n))
+ *                                          + lambda d_n ) ( 1[v = y_n] - p_s(v) ),
+ *                         which needs the student row only.
+ */
+typedef enum { FOPD_LOSS_FULL_KL = 0, FOPD_LOSS_SAMPLED_KL = 1 } fopd_loss_kind;
+
 typedef enum {
   FOPD_OK = 0,
   FOPD_ERR_NULL = -1,   /* a required pointer is NULL                          */
@@ -86,7 +104,8 @@ typedef enum {
   FOPD_ERR_PARAM = -5,  /* alpha/beta negative or a parameter not finite        */
   FOPD_ERR_CUDA = -6,   /* a CUDA runtime call failed (launch, allocation)      */
   FOPD_ERR_ALIAS = -7,  /* dlogits overlaps student or teacher                  */
-  FOPD_ERR_DEVICE = -8  /* fopd_check_status: the device status word is non-zero */
+  FOPD_ERR_DEVICE = -8, /* fopd_check_status: the device status word is non-zero */
+  FOPD_ERR_KIND = -9    /* loss_kind unknown, or not supported by this entry point */
 } fopd_status;
 
 /* Bits ORed into the device status word. */
@@ -123,12 +142,13 @@ typedef struct {
   int64_t vocab;
   int64_t row_stride;
   int32_t dtype;              /* fopd_dtype                                     */
+  int32_t loss_kind;          /* fopd_loss_kind; the same for every chunk and call of a batch */
 } fopd_chunk;
 
 /* Columns of the per-row workspace row_ws[n_rows, 4] (fp32). */
 #define FOPD_WS_LSE_S 0
 #define FOPD_WS_LSE_T 1
-#define FOPD_WS_KL 2
+#define FOPD_WS_KL 2 /* FOPD_LOSS_SAMPLED_KL: log p_s(y_n) - log p_t(y_n) instead */
 #define FOPD_WS_D 3 /* d_n = lp_s - b_n = log rho_n */
 
 /* Columns of acc[B, 4] (fp64): aligned-row count, sum of k3, sum of kl, rows seen. */
@@ -143,7 +163,8 @@ typedef struct {
  * the stored token, the Eq. 12 token loss and the Eq. 10 drift integrand.
  *
  *   lp_s, lp_t, kl, ratio  [n_rows] fp32 outputs, any may be NULL.  Rows with
- *                          mask = 0 or a bad id get exactly 0.
+ *                          mask = 0 or a bad id get exactly 0.  kl is the token loss
+ *                          in the chunk's loss_kind (and so is the sum in acc).
  *   row_ws                 optional [n_rows, 4] fp32 output (columns above),
  *                          16-byte aligned; pass it to fopd_loss_fwd_bwd for
  *                          the same chunk to let that call skip its own
@@ -171,12 +192,13 @@ int fopd_token_stats(const fopd_chunk *chunk /* HOST */, int32_t B, float *lp_s,
  *
  * Same arguments, outputs and results as fopd_token_stats without the row_ws
  * parameter: the per-row scratch lives in a fixed array compiled into the
- * library, FOPD_STATIC_MAX_ROWS * 16 bytes = 1 MiB on every GPU that loads the
- * library, held until the process exits.  The call makes no cudaMalloc,
+ * library, FOPD_STATIC_MAX_ROWS * 16 bytes = 1 MiB for the rows plus
+ * FOPD_STATIC_MAX_SAMPLES * 16 bytes = 256 KiB for the samples' row ranges, on
+ * every GPU that loads the library, held until the process exits.  The call makes no cudaMalloc,
  * cudaFree or other allocating call.
  *
- *   - chunk->n_rows > FOPD_STATIC_MAX_ROWS returns FOPD_ERR_SIZE and enqueues
- *     nothing; split the chunk.
+ *   - chunk->n_rows > FOPD_STATIC_MAX_ROWS or B > FOPD_STATIC_MAX_SAMPLES returns
+ *     FOPD_ERR_SIZE and enqueues nothing; split the chunk (or the batch).
  *   - The first call on each device looks the array's device address up
  *     (cudaGetSymbolAddress, with that device current) and caches it.  With
  *     CUDA's lazy module loading that first call is also what loads the part of
@@ -185,13 +207,14 @@ int fopd_token_stats(const fopd_chunk *chunk /* HOST */, int32_t B, float *lp_s,
  *     outside any stream capture and before the rest of the device's memory is
  *     handed to another allocator.  If it fails it returns FOPD_ERR_CUDA and
  *     can be repeated.
- *   - All calls on a device share the one array, which still holds the previous
- *     call's values.  Nothing has to be cleared: each call overwrites the
- *     entries of all its rows before it reads them.  Two calls whose kernels can
+ *   - All calls on a device share the two arrays, which still hold the previous
+ *     call's values.  The caller has nothing to clear: each call overwrites the
+ *     entries of all its rows and samples before it reads them.  Two calls whose kernels can
  *     overlap on the GPU (different streams, or the same entry point from two
  *     threads) race on the array; order them on one stream.
  */
 #define FOPD_STATIC_MAX_ROWS 65536
+#define FOPD_STATIC_MAX_SAMPLES 16384
 int fopd_token_stats_static(const fopd_chunk *chunk /* HOST */, int32_t B, float *lp_s,
                             float *lp_t, float *kl, float *ratio, double *acc,
                             int32_t *status, void *stream);
@@ -225,7 +248,9 @@ int fopd_sample_freshness(const double *acc, const int32_t *staleness,
  *   dlogits[n,v] = coef_i { p_s(v) [ (log p_s(v) - log p_t(v)) - kl_n ]
  *                           + lambda rho_n d_n ( 1[v = y_n] - p_s(v) ) }
  *
- * Every other row of dlogits (masked, padded, bad id, gated or invalid sample)
+ * (chunk->loss_kind = FOPD_LOSS_SAMPLED_KL: the formula given with fopd_loss_kind; with
+ * row_ws that call is one pass that reads S and writes dlogits, without it the statistics
+ * sweep runs first.)  Every other row of dlogits (masked, padded, bad id, gated or invalid sample)
  * is written as +0 and its logits are not read.  The per-sample sums of kl and
  * k3 over the rows this call differentiated are ADDED to loss_acc.
  *
@@ -344,6 +369,7 @@ int fopd_refresh_decision(const float *f, const float *m_roll, const float *m_su
  * split over a partition of the vocabulary: with m_k = max, Z_k = sum e^{x - m_k}
  * and A_k = sum e^{s - m_k}(s - t) over part k,
  *   lse = log sum_k Z_k e^{m_k},   sum_v p_s(v)(s_v - t_v) = sum_k A_k e^{m_k} / sum_k Z_k e^{m_k}.
+ * These entry points take FOPD_LOSS_FULL_KL only (FOPD_ERR_KIND otherwise).
  * Calling sequence on every holder, per chunk: fopd_shard_stats -> exchange the
  * partial sums so that every holder has all parts (the caller's job: an all-gather
  * of [n_rows, 8] floats per holder; the library makes no collective call) ->

@@ -15,6 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libfopd.so")
 
 FOPD_BF16, FOPD_F32 = 0, 1
+LOSS_FULL_KL, LOSS_SAMPLED_KL = 0, 1  # forms of the token loss (fopd_loss_kind)
 
 EXPORTS = (
     "fopd_token_stats", "fopd_sample_freshness", "fopd_loss_fwd_bwd", "fopd_loss_finalize",
@@ -41,7 +42,7 @@ class fopd_chunk(ctypes.Structure):
         ("student", ctypes.c_void_p), ("teacher", ctypes.c_void_p), ("behav_logprob", ctypes.c_void_p),
         ("tokens", ctypes.c_void_p), ("mask", ctypes.c_void_p), ("sample_id", ctypes.c_void_p),
         ("n_rows", ctypes.c_int64), ("vocab", ctypes.c_int64), ("row_stride", ctypes.c_int64),
-        ("dtype", ctypes.c_int32),
+        ("dtype", ctypes.c_int32), ("loss_kind", ctypes.c_int32),
     ]
 
 
@@ -132,6 +133,7 @@ class Chunk:
     mask: torch.Tensor  # [n] uint8
     sample_id: torch.Tensor  # [n] int32
     vocab: int | None = None  # columns in use; defaults to student.shape[1]
+    loss_kind: int = LOSS_FULL_KL
 
     def c_struct(self) -> fopd_chunk:
         S, T = self.student, self.teacher
@@ -146,7 +148,7 @@ class Chunk:
             S.data_ptr(), T.data_ptr(), self.behav_logprob.data_ptr(), self.tokens.data_ptr(),
             self.mask.data_ptr(), self.sample_id.data_ptr(), n, self.vocab or S.shape[1],
             S.stride(0) if n > 1 else max(S.stride(0), S.shape[1]),
-            FOPD_BF16 if S.dtype == torch.bfloat16 else FOPD_F32,
+            FOPD_BF16 if S.dtype == torch.bfloat16 else FOPD_F32, int(self.loss_kind),
         )
 
 
@@ -159,6 +161,7 @@ def fopd_token_stats(chunk: Chunk, B: int, acc, *, lp_s=None, lp_t=None, kl=None
 
 
 STATIC_MAX_ROWS = 65536
+STATIC_MAX_SAMPLES = 16384
 
 
 def fopd_token_stats_static(chunk: Chunk, B: int, acc, *, lp_s=None, lp_t=None, kl=None, ratio=None,
@@ -265,7 +268,7 @@ def fopd_shard_merge(partials, behav_logprob, tokens, mask, sample_id, vocab_tot
     assert partials.dtype == torch.float32 and partials.is_contiguous() and partials.dim() == 3
     assert partials.shape[1] == n and partials.shape[2] == 8
     rows = fopd_chunk(None, None, behav_logprob.data_ptr(), tokens.data_ptr(), mask.data_ptr(),
-                      sample_id.data_ptr(), n, int(vocab_total), int(vocab_total), FOPD_F32)
+                      sample_id.data_ptr(), n, int(vocab_total), int(vocab_total), FOPD_F32, LOSS_FULL_KL)
     _check(lib().fopd_shard_merge(_ptr(partials), partials.shape[0], ctypes.byref(rows), B, _ptr(lp_s), _ptr(lp_t),
                                   _ptr(kl), _ptr(ratio), _ptr(row_ws), _ptr(acc), _ptr(status), _stream(stream)),
            "fopd_shard_merge")

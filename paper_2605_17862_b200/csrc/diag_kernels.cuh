@@ -138,13 +138,12 @@ __global__ void __launch_bounds__(kDiagThreads, 4)
 // per sample, fixed strided partials, fixed tree, fp64), accumulates across chunks.
 static __global__ void __launch_bounds__(kSegThreads)
     divergence_reduce_kernel(const int32_t *sid, const uint8_t *mask, int64_t n_rows, const float2 *vals,
-                             double *out) {
+                             const unsigned long long *bounds, double *out) {
   __shared__ double sh[3][kSegThreads];
-  __shared__ int64_t range_sh[2];
   const int32_t i = blockIdx.x;
-  int64_t lo, hi;
-  sample_row_range(sid, n_rows, i, range_sh, lo, hi);
-  if (lo >= hi) return;
+  const unsigned long long lo_u = bounds[2 * (int64_t)i], hi_u = bounds[2 * (int64_t)i + 1];
+  if (lo_u >= hi_u) return;
+  const int64_t lo = (int64_t)lo_u, hi = (int64_t)hi_u;
   double cnt = 0.0, skl = 0.0, sen = 0.0;
   for (int64_t n = lo + threadIdx.x; n < hi; n += kSegThreads) {
     if (sid[n] != i || mask[n] == 0) continue;

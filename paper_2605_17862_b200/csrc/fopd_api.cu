@@ -235,6 +235,7 @@ const char *fopd_strerror(int code) {
     case FOPD_ERR_CUDA: return "a CUDA runtime call failed";
     case FOPD_ERR_ALIAS: return "dlogits overlaps student or teacher";
     case FOPD_ERR_DEVICE: return "device status word is non-zero (bad token/sample id, staleness, length or timeout)";
+    case FOPD_ERR_KIND: return "loss_kind unknown or not supported by this entry point";
     default: return "unknown fopd status";
   }
 }
@@ -247,17 +248,21 @@ int fopd_token_stats(const fopd_chunk *chunk, int32_t B, float *lp_s, float *lp_
   if (row_ws && !aligned16(row_ws)) return FOPD_ERR_ALIGN;
   if (chunk->n_rows == 0) return FOPD_OK;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  float *ws = row_ws;
-  if (!ws) {
-    if ((rc = scratch_alloc(reinterpret_cast<void **>(&ws), (size_t)chunk->n_rows * 4 * sizeof(float), st)) != FOPD_OK)
-      return rc;
-  }
+  // one temporary: the samples' row ranges, then the row statistics if the caller keeps none
+  const size_t bb = (bounds_bytes(B) + 255) & ~size_t(255);
+  char *tmp = nullptr;
+  if ((rc = scratch_alloc(reinterpret_cast<void **>(&tmp), bb + (row_ws ? 0 : (size_t)chunk->n_rows * 4 * sizeof(float)), st)) !=
+      FOPD_OK)
+    return rc;
+  unsigned long long *bounds = reinterpret_cast<unsigned long long *>(tmp);
+  float *ws = row_ws ? row_ws : reinterpret_cast<float *>(tmp + bb);
   rc = launch_stats(chunk, B, lp_s, lp_t, kl, ratio, ws, status, st);
+  if (rc == FOPD_OK) rc = launch_sample_bounds(chunk->sample_id, chunk->n_rows, B, bounds, st);
   if (rc == FOPD_OK) {
-    segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(to_dev(chunk), B, ws, nullptr, 0, acc);
+    segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(to_dev(chunk), B, ws, nullptr, 0, bounds, acc);
     rc = launch_ok();
   }
-  if (!row_ws && cudaFreeAsync(ws, st) != cudaSuccess) rc = FOPD_ERR_CUDA;
+  if (cudaFreeAsync(tmp, st) != cudaSuccess) rc = FOPD_ERR_CUDA;
   return rc;
 }
 
@@ -292,17 +297,26 @@ int fopd_loss_fwd_bwd(const fopd_chunk *chunk, int32_t B, const float *coef, con
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const ChunkDev d = to_dev(chunk);
   const float *ws = row_ws;
-  float *tmp = nullptr;
+  // one temporary: the samples' row ranges, then (without cached statistics) [n_rows, 4] row
+  // statistics and [n_rows] row weights
+  const size_t bb = (bounds_bytes(B) + 255) & ~size_t(255);
+  char *blk = nullptr;
+  if ((rc = scratch_alloc(reinterpret_cast<void **>(&blk), bb + (ws ? 0 : (size_t)chunk->n_rows * 5 * sizeof(float)), st)) !=
+      FOPD_OK)
+    return rc;
+  unsigned long long *bounds = reinterpret_cast<unsigned long long *>(blk);
   bool grad_done = false;
   if (!ws) {
-    // No cached statistics.  Preferred: the on-chip kernel, which does the reduction sweep
-    // and the gradient sweep from shared memory and leaves the row statistics in tmp.
-    // Shapes it cannot take fall back to the statistics sweep + streaming gradient pair.
-    if ((rc = scratch_alloc(reinterpret_cast<void **>(&tmp), (size_t)chunk->n_rows * 5 * sizeof(float), st)) != FOPD_OK)
-      return rc;
+    // No cached statistics.  Preferred: the on-chip kernel, which forms the sums and the
+    // gradient of a row while it is on chip and leaves the row statistics in tmp.  Shapes it
+    // cannot take fall back to the statistics sweep + streaming gradient pair.
+    float *tmp = reinterpret_cast<float *>(blk + bb);
     ws = tmp;
-    rc = chunk->dtype == FOPD_BF16 ? launch_fused<FOPD_BF16>(chunk, B, coef, p.lambda, dlogits, tmp, status, st)
-                                   : launch_fused<FOPD_F32>(chunk, B, coef, p.lambda, dlogits, tmp, status, st);
+    // (the sampled-token form needs no teacher row for its gradient: statistics sweep + one pass)
+    rc = chunk->loss_kind != FOPD_LOSS_FULL_KL
+             ? kNotApplicable
+             : chunk->dtype == FOPD_BF16 ? launch_fused<FOPD_BF16>(chunk, B, coef, p.lambda, dlogits, tmp, status, st)
+                                         : launch_fused<FOPD_F32>(chunk, B, coef, p.lambda, dlogits, tmp, status, st);
     if (rc == FOPD_OK) grad_done = true;
     else if (rc == kNotApplicable)
       rc = launch_stats(chunk, B, nullptr, nullptr, nullptr, nullptr, tmp, status, st);
@@ -310,7 +324,13 @@ int fopd_loss_fwd_bwd(const fopd_chunk *chunk, int32_t B, const float *coef, con
   if (rc == FOPD_OK && !grad_done) {
     const unsigned grid = row_grid(chunk->n_rows);
     const bool short_row = chunk->vocab / (chunk->dtype == FOPD_BF16 ? 8 : 4) < kShortRowVecs;
-#define FOPD_LAUNCH_GRAD(DT, T) grad_stream_kernel<DT, T><<<grid, T, 0, st>>>(d, B, coef, ws, p.lambda, dlogits)
+#define FOPD_LAUNCH_GRAD(DT, T)                                                          \
+  do {                                                                                     \
+    if (chunk->loss_kind == FOPD_LOSS_SAMPLED_KL)                                          \
+      grad_sampled_kernel<DT, T><<<grid, T, 0, st>>>(d, B, coef, ws, p.lambda, dlogits);   \
+    else                                                                                   \
+      grad_stream_kernel<DT, T><<<grid, T, 0, st>>>(d, B, coef, ws, p.lambda, dlogits);    \
+  } while (0)
     if (chunk->dtype == FOPD_BF16) {
       if (short_row) FOPD_LAUNCH_GRAD(FOPD_BF16, kGradThreadsShortRow);
       else FOPD_LAUNCH_GRAD(FOPD_BF16, kGradThreads);
@@ -321,11 +341,12 @@ int fopd_loss_fwd_bwd(const fopd_chunk *chunk, int32_t B, const float *coef, con
 #undef FOPD_LAUNCH_GRAD
     rc = launch_ok();
   }
+  if (rc == FOPD_OK) rc = launch_sample_bounds(chunk->sample_id, chunk->n_rows, B, bounds, st);
   if (rc == FOPD_OK) {
-    segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(d, B, ws, coef, 1, loss_acc);
+    segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(d, B, ws, coef, 1, bounds, loss_acc);
     rc = launch_ok();
   }
-  if (tmp && cudaFreeAsync(tmp, st) != cudaSuccess) rc = FOPD_ERR_CUDA;
+  if (cudaFreeAsync(blk, st) != cudaSuccess) rc = FOPD_ERR_CUDA;
   return rc;
 }
 

@@ -18,9 +18,13 @@ int fopd_row_divergence(const void *first, const void *second, const uint8_t *ma
   const int64_t esz = dtype == FOPD_BF16 ? 2 : 4;
   if (!aligned16(first) || !aligned16(second) || (row_stride * esz) % 16 != 0) return FOPD_ERR_ALIGN;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  float2 *vals = nullptr;
-  int rc = scratch_alloc(reinterpret_cast<void **>(&vals), (size_t)n_rows * sizeof(float2), st);
+  // one temporary: the samples' row ranges, then {kl, entropy} of every row
+  const size_t bb = (bounds_bytes(B) + 255) & ~size_t(255);
+  char *tmp = nullptr;
+  int rc = scratch_alloc(reinterpret_cast<void **>(&tmp), bb + (size_t)n_rows * sizeof(float2), st);
   if (rc != FOPD_OK) return rc;
+  unsigned long long *bounds = reinterpret_cast<unsigned long long *>(tmp);
+  float2 *vals = reinterpret_cast<float2 *>(tmp + bb);
   const unsigned grid = row_grid(n_rows);
   if (dtype == FOPD_BF16)
     row_divergence_kernel<FOPD_BF16><<<grid, kDiagThreads, 0, st>>>(first, second, mask, sample_id, n_rows, vocab,
@@ -29,11 +33,12 @@ int fopd_row_divergence(const void *first, const void *second, const uint8_t *ma
     row_divergence_kernel<FOPD_F32><<<grid, kDiagThreads, 0, st>>>(first, second, mask, sample_id, n_rows, vocab,
                                                                  row_stride, B, kl, entropy, vals, status);
   rc = launch_ok();
+  if (rc == FOPD_OK) rc = launch_sample_bounds(sample_id, n_rows, B, bounds, st);
   if (rc == FOPD_OK) {
-    divergence_reduce_kernel<<<B, kSegThreads, 0, st>>>(sample_id, mask, n_rows, vals, acc);
+    divergence_reduce_kernel<<<B, kSegThreads, 0, st>>>(sample_id, mask, n_rows, vals, bounds, acc);
     rc = launch_ok();
   }
-  if (cudaFreeAsync(vals, st) != cudaSuccess) rc = FOPD_ERR_CUDA;
+  if (cudaFreeAsync(tmp, st) != cudaSuccess) rc = FOPD_ERR_CUDA;
   return rc;
 }
 

@@ -10,6 +10,7 @@ namespace {
 int check_shard(const fopd_chunk *shard, int64_t vocab_offset, int64_t vocab_total) {
   int rc = check_chunk(shard, 1);
   if (rc != FOPD_OK) return rc;
+  if (shard->loss_kind != FOPD_LOSS_FULL_KL) return FOPD_ERR_KIND;
   if (vocab_offset < 0 || vocab_total > (int64_t)1 << 30 || vocab_offset + shard->vocab > vocab_total)
     return FOPD_ERR_SIZE;
   return FOPD_OK;
@@ -18,6 +19,7 @@ int check_shard(const fopd_chunk *shard, int64_t vocab_offset, int64_t vocab_tot
 // The per-row side arrays of a chunk without its logits, judged against the full vocabulary.
 int check_rows(const fopd_chunk *rows, int32_t B) {
   if (!rows) return FOPD_ERR_NULL;
+  if (rows->loss_kind != FOPD_LOSS_FULL_KL) return FOPD_ERR_KIND;
   if (rows->n_rows < 0 || rows->vocab <= 0 || rows->vocab > (int64_t)1 << 30 || B <= 0) return FOPD_ERR_SIZE;
   if (rows->n_rows > 0 && (!rows->behav_logprob || !rows->tokens || !rows->mask || !rows->sample_id))
     return FOPD_ERR_NULL;
@@ -66,8 +68,7 @@ int fopd_shard_merge(const float *partials, int32_t n_parts, const fopd_chunk *r
   shard_merge_kernel<<<(unsigned)((rows->n_rows + 255) / 256), 256, 0, st>>>(partials, n_parts, d, B, lp_s, lp_t, kl,
                                                                            ratio, row_ws, status);
   if ((rc = launch_ok()) != FOPD_OK) return rc;
-  segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(d, B, row_ws, nullptr, 0, acc);
-  return launch_ok();
+  return launch_segment_reduce(d, B, row_ws, nullptr, 0, acc, st);
 }
 
 int fopd_shard_loss_fwd_bwd(const fopd_chunk *shard, int64_t vocab_offset, int64_t vocab_total, int32_t B,
@@ -106,8 +107,7 @@ int fopd_shard_loss_fwd_bwd(const fopd_chunk *shard, int64_t vocab_offset, int64
   if (loss_acc) {  // the sums do not depend on the shard: every holder gets the same, or one holder asks
     ChunkDev whole = d;
     whole.vocab = vocab_total;
-    segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(whole, B, row_ws, coef, 1, loss_acc);
-    rc = launch_ok();
+    rc = launch_segment_reduce(whole, B, row_ws, coef, 1, loss_acc, st);
   }
   return rc;
 }

@@ -12,15 +12,18 @@ using namespace fopd;
 // process exits.  In host code this name is only a handle for the symbol, not
 // a device address: the address is looked up once per device below.
 static __device__ __align__(256) float g_static_row_ws[(size_t)FOPD_STATIC_MAX_ROWS * 4];
+// Row range of every sample in the chunk, for up to FOPD_STATIC_MAX_SAMPLES samples (256 KiB).
+static __device__ __align__(256) unsigned long long g_static_bounds[(size_t)FOPD_STATIC_MAX_SAMPLES * 2];
 
 namespace {
 
 std::mutex g_setup_mutex;
 float *g_static_row_ws_addr[kMaxDevices] = {};
+unsigned long long *g_static_bounds_addr[kMaxDevices] = {};
 
 // Device address of the scratch array on the current device.  Looked up with
 // cudaGetSymbolAddress the first time this device calls in, then cached.
-int static_scratch(float **out) {
+int static_scratch(float **out, unsigned long long **bounds_out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return FOPD_ERR_CUDA;
   std::lock_guard<std::mutex> lock(g_setup_mutex);
@@ -30,9 +33,16 @@ int static_scratch(float **out) {
       (void)cudaGetLastError();  // leave no sticky-looking error behind for the caller's next check
       return FOPD_ERR_CUDA;
     }
+    unsigned long long *bptr = nullptr;
+    if (cudaGetSymbolAddress(reinterpret_cast<void **>(&bptr), g_static_bounds) != cudaSuccess || !bptr) {
+      (void)cudaGetLastError();
+      return FOPD_ERR_CUDA;
+    }
     g_static_row_ws_addr[dev] = ptr;
+    g_static_bounds_addr[dev] = bptr;
   }
   *out = g_static_row_ws_addr[dev];
+  *bounds_out = g_static_bounds_addr[dev];
   return FOPD_OK;
 }
 
@@ -44,16 +54,19 @@ extern "C" int fopd_token_stats_static(const fopd_chunk *chunk, int32_t B, float
   int rc = check_chunk(chunk, B);
   if (rc != FOPD_OK) return rc;
   if (!acc) return FOPD_ERR_NULL;
-  if (chunk->n_rows > FOPD_STATIC_MAX_ROWS) return FOPD_ERR_SIZE;
+  if (chunk->n_rows > FOPD_STATIC_MAX_ROWS || B > FOPD_STATIC_MAX_SAMPLES) return FOPD_ERR_SIZE;
   if (chunk->n_rows == 0) return FOPD_OK;
   float *ws = nullptr;
-  if ((rc = static_scratch(&ws)) != FOPD_OK) return rc;
+  unsigned long long *bounds = nullptr;
+  if ((rc = static_scratch(&ws, &bounds)) != FOPD_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // The sweep writes all four scratch values of every row of the chunk (zeros
-  // for rows that are not aligned) before the reduction reads them, so nothing
-  // left over from an earlier call is ever read and nothing needs clearing.
+  // for rows that are not aligned) before the reduction reads them, and the row
+  // ranges of all B samples are reset before they are filled in, so nothing
+  // left over from an earlier call is ever read.
   rc = launch_stats(chunk, B, lp_s, lp_t, kl, ratio, ws, status, st);
   if (rc != FOPD_OK) return rc;
-  segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(to_dev(chunk), B, ws, nullptr, 0, acc);
+  if ((rc = launch_sample_bounds(chunk->sample_id, chunk->n_rows, B, bounds, st)) != FOPD_OK) return rc;
+  segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(to_dev(chunk), B, ws, nullptr, 0, bounds, acc);
   return launch_ok();
 }

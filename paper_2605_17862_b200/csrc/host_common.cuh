@@ -14,6 +14,7 @@ static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t
 static inline int check_chunk(const fopd_chunk *c, int32_t B) {
   if (!c) return FOPD_ERR_NULL;
   if (c->dtype != FOPD_BF16 && c->dtype != FOPD_F32) return FOPD_ERR_DTYPE;
+  if (c->loss_kind != FOPD_LOSS_FULL_KL && c->loss_kind != FOPD_LOSS_SAMPLED_KL) return FOPD_ERR_KIND;
   if (c->n_rows < 0 || c->vocab <= 0 || c->row_stride < c->vocab || B <= 0) return FOPD_ERR_SIZE;
   if (c->vocab > (int64_t)1 << 30 || c->n_rows > (int64_t)1 << 40) return FOPD_ERR_SIZE;
   if (c->n_rows == 0) return FOPD_OK;
@@ -36,6 +37,7 @@ static inline ChunkDev to_dev(const fopd_chunk *c) {
   d.n_rows = c->n_rows;
   d.vocab = c->vocab;
   d.stride = c->row_stride;
+  d.kind = c->loss_kind;
   return d;
 }
 
@@ -96,6 +98,31 @@ static inline int scratch_release() {
   std::lock_guard<std::mutex> lock(sp.mu);
   if (!sp.pools[dev]) return FOPD_OK;
   return cudaMemPoolTrimTo(sp.pools[dev], 0) == cudaSuccess ? FOPD_OK : FOPD_ERR_CUDA;
+}
+
+// Enqueues the pass that finds every sample's row range in a chunk (bounds: [B, 2] 64-bit).
+static inline int launch_sample_bounds(const int32_t *sid, int64_t n_rows, int32_t B, unsigned long long *bounds,
+                                       cudaStream_t st) {
+  sample_bounds_init_kernel<<<(unsigned)((B + 255) / 256), 256, 0, st>>>(B, bounds);
+  if (n_rows > 0) sample_bounds_kernel<<<(unsigned)((n_rows + 255) / 256), 256, 0, st>>>(sid, n_rows, B, bounds);
+  return launch_ok();
+}
+static inline size_t bounds_bytes(int32_t B) { return (size_t)B * 2 * sizeof(unsigned long long); }
+
+// The per-sample reduction of a chunk's row statistics with its row ranges in a temporary of
+// the library's pool.  mode 0: acc[B,4] +=; mode 1: loss_acc[B,2] += (see segment_reduce_kernel).
+static inline int launch_segment_reduce(const ChunkDev &d, int32_t B, const float *row_ws, const float *coef, int mode,
+                                        double *out, cudaStream_t st) {
+  unsigned long long *bounds = nullptr;
+  int rc = scratch_alloc(reinterpret_cast<void **>(&bounds), bounds_bytes(B), st);
+  if (rc != FOPD_OK) return rc;
+  rc = launch_sample_bounds(d.sid, d.n_rows, B, bounds, st);
+  if (rc == FOPD_OK) {
+    segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(d, B, row_ws, coef, mode, bounds, out);
+    rc = launch_ok();
+  }
+  if (cudaFreeAsync(bounds, st) != cudaSuccess) rc = FOPD_ERR_CUDA;
+  return rc;
 }
 
 // One CTA per row.

@@ -86,7 +86,7 @@ static __global__ void __launch_bounds__(256)
     zero_row_outputs(n, lp_s, lp_t, kl, ratio, row_ws);
     return;
   }
-  finish_row<FOPD_F32>(n, r, sy, ty, c.behav[n], lp_s, lp_t, kl, ratio, row_ws);
+  finish_row<FOPD_F32>(n, r, sy, ty, c.behav[n], FOPD_LOSS_FULL_KL, lp_s, lp_t, kl, ratio, row_ws);
 }
 
 // Gradient of one shard's columns from the merged row statistics.  c is the shard's view

@@ -28,6 +28,7 @@ struct ChunkDev {
   const uint8_t *mask;
   const int32_t *sid;
   int64_t n_rows, vocab, stride;
+  int kind;  // fopd_loss_kind
 };
 
 // Is row n aligned (counts towards U_i)?  Records bad ids in the status word.
@@ -53,8 +54,8 @@ __device__ __forceinline__ bool row_is_aligned(const ChunkDev &c, int64_t n, int
 // Turns the finished accumulators of a row into the quantities of Sec. 4.1 /
 // Eq. 10 / Eq. 12 and writes the per-row outputs.  Called by one thread.
 template <int DT>
-__device__ __forceinline__ void finish_row(int64_t n, const RowAcc &r, float sy, float ty, float b, float *lp_s,
-                                           float *lp_t, float *kl_out, float *ratio, float *row_ws) {
+__device__ __forceinline__ void finish_row(int64_t n, const RowAcc &r, float sy, float ty, float b, int kind,
+                                           float *lp_s, float *lp_t, float *kl_out, float *ratio, float *row_ws) {
   // log of the partition sums in full precision (logf, not the fast intrinsic)
   // differences are formed from the maxima and the logs separately, so that they do not inherit
   // the rounding of a large log-normaliser
@@ -65,9 +66,13 @@ __device__ __forceinline__ void finish_row(int64_t n, const RowAcc &r, float sy,
   const float d = lps - b;
   if (lp_s) lp_s[n] = lps;
   if (lp_t) lp_t[n] = lpt;
-  if (kl_out) kl_out[n] = kl;
-  if (ratio) ratio[n] = expf(d);  // fp32 is ample for the reported ratio; the drift integrand is formed in fp64 from d
-  reinterpret_cast<float4 *>(row_ws)[n] = make_float4(ls, lt, kl, d);
+  const float rho = expf(d);  // fp32 is ample for the reported ratio; the drift integrand is formed in fp64 from d
+  // sampled-token form of Eq. 12's loss: rho (lp_s - lp_t) on the stored token; the workspace
+  // keeps the log-ratio, which the gradient takes as a constant
+  const float log_ratio = lps - lpt;
+  if (kl_out) kl_out[n] = kind == FOPD_LOSS_SAMPLED_KL ? rho * log_ratio : kl;
+  if (ratio) ratio[n] = rho;
+  reinterpret_cast<float4 *>(row_ws)[n] = make_float4(ls, lt, kind == FOPD_LOSS_SAMPLED_KL ? log_ratio : kl, d);
 }
 
 __device__ __forceinline__ void zero_row_outputs(int64_t n, float *lp_s, float *lp_t, float *kl_out,
@@ -141,7 +146,7 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads)
     const char *trow = reinterpret_cast<const char *>(c.teacher) + n * c.stride * E::kBytes;
     RowAcc acc = sweep_row_global<DT, kThreads>(srow, trow, c.vocab);
     acc = block_reduce<kThreads>(acc, scratch[par]);
-    if (threadIdx.x == 0) finish_row<DT>(n, acc, sy, ty, b, lp_s, lp_t, kl, ratio, row_ws);
+    if (threadIdx.x == 0) finish_row<DT>(n, acc, sy, ty, b, c.kind, lp_s, lp_t, kl, ratio, row_ws);
     par ^= 1;
   }
 }
@@ -260,44 +265,104 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads)
   }
 }
 
+// Row range of every sample within a chunk, found in one pass over the rows: bounds[2i] =
+// first row whose sample id is i, bounds[2i + 1] = one past the last such row (first >= last:
+// the sample has no row in this chunk).  Rows of a sample are contiguous, so a row starts a
+// run where its id differs from the row before and ends one where it differs from the row
+// after; minimum / maximum over the runs keep the result unique when an out-of-range id sits
+// in the middle of a sample (the rows in between are skipped by their own id).
+static __global__ void __launch_bounds__(256) sample_bounds_init_kernel(int32_t B, unsigned long long *bounds) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < B) {
+    bounds[2 * i] = ~0ull;
+    bounds[2 * i + 1] = 0ull;
+  }
+}
+static __global__ void __launch_bounds__(256)
+    sample_bounds_kernel(const int32_t *sid, int64_t n_rows, int32_t B, unsigned long long *bounds) {
+  const int64_t n = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (n >= n_rows) return;
+  const int32_t s = sid[n];
+  if (s < 0 || s >= B) return;
+  if (n == 0 || sid[n - 1] != s) atomicMin(&bounds[2 * (int64_t)s], (unsigned long long)n);
+  if (n == n_rows - 1 || sid[n + 1] != s) atomicMax(&bounds[2 * (int64_t)s + 1], (unsigned long long)(n + 1));
+}
+
+// a8 for the sampled-token form of the loss, with cached row statistics: one streaming pass
+// that reads S and writes dS.  For a differentiated row
+//   dS_v = coef rho (r + lambda d) (1[v = y] - p_s(v)),   r = lp_s - lp_t (constant), d = lp_s - b,
+// i.e. -G cp_v + [v == y] G coef with cp_v = coef p_s(v) = 2^(s_v*log2e + e0), G = rho (r + lambda d).
+template <int DT, int kThreads>
+__global__ void __launch_bounds__(kThreads, 1024 / kThreads)
+    grad_sampled_kernel(ChunkDev c, int32_t B, const float *coef, const float *row_ws, float lambda, void *dlogits) {
+  using E = Elem<DT>;
+  constexpr int P = E::kPerVec;
+  for (int64_t n = blockIdx.x; n < c.n_rows; n += gridDim.x) {
+    char *orow = reinterpret_cast<char *>(dlogits) + n * c.stride * E::kBytes;
+    const int32_t sid = c.sid[n], y = c.tokens[n];
+    const uint8_t m = c.mask[n];
+    const float4 ws = reinterpret_cast<const float4 *>(row_ws)[n];
+    const bool sid_ok = sid >= 0 && sid < B;
+    float cf = sid_ok ? coef[sid] : 0.f;
+    if (m == 0 || y < 0 || y >= c.vocab) cf = 0.f;
+    if (!(cf > 0.f)) {
+      zero_fill_row<DT, kThreads>(orow, c.vocab);
+      continue;
+    }
+    const float d = ws.w, G = expf(d) * (ws.z + lambda * d);
+    const float e0 = log2f(cf) - ws.x * kLog2e, negG = -G, cg = cf * G;
+    const char *srow = reinterpret_cast<const char *>(c.student) + n * c.stride * E::kBytes;
+    const int64_t V = c.vocab, nvec = V / P;
+    const uint4 *s4 = reinterpret_cast<const uint4 *>(srow);
+    uint4 *o4 = reinterpret_cast<uint4 *>(orow);
+    auto one = [&](const uint4 &sv) {
+      float s[P], o[P];
+      E::unpack(sv, s);
+#pragma unroll
+      for (int i = 0; i < P; ++i) o[i] = ex2(fmaf(s[i], kLog2e, e0)) * negG;
+      return E::pack(o);
+    };
+    int64_t i = threadIdx.x;
+    for (; i + (kUnroll - 1) * kThreads < nvec; i += kUnroll * kThreads) {
+      uint4 a[kUnroll];
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) a[u] = ld_stream(s4 + i + u * kThreads);
+#pragma unroll
+      for (int u = 0; u < kUnroll; ++u) st_stream(o4 + i + u * kThreads, one(a[u]));
+    }
+    for (; i < nvec; i += kThreads) st_stream(o4 + i, one(ld_stream(s4 + i)));
+    // the stored token's element: rewritten with its extra term by the thread that stored its vector
+    const int64_t yv = y / P;
+    if (yv < nvec && (int)(yv % kThreads) == (int)threadIdx.x) {
+      const float s = E::load1(srow, y);
+      E::store1(orow, y, fmaf(ex2(fmaf(s, kLog2e, e0)), negG, cg));
+    }
+    const int64_t tail = nvec * P + threadIdx.x;
+    if (tail < V) {
+      const float s = E::load1(srow, tail);
+      float o = ex2(fmaf(s, kLog2e, e0)) * negG;
+      if (tail == y) o = fmaf(ex2(fmaf(s, kLog2e, e0)), negG, cg);
+      E::store1(orow, tail, o);
+    }
+  }
+}
+
 // a5: deterministic segmented reduction of per-row statistics into per-sample
-// sums.  One block per sample; the block finds its (contiguous) row range by a
-// parallel scan for the two places where the non-decreasing sample_id array
-// crosses its id (independent loads: a binary search is a chain of ~30 dependent
-// ones), every thread sums a
+// sums.  One block per sample over the sample's row range; every thread sums a
 // fixed strided subset in fp64 and a fixed tree combines them, so a rerun
 // reproduces the bits.  mode 0: acc[B,4] += {cnt, sum k3, sum kl, rows}.
 // mode 1: loss_acc[B,2] += {sum kl, sum k3} over rows of samples with coef > 0.
 constexpr int kSegThreads = 1024;
 
-// First row with sample id >= key and first row with id >= key + 1 (n where there is none),
-// found by all threads of the block together; valid in every thread after the call.
-__device__ __forceinline__ void sample_row_range(const int32_t *sid, int64_t n, int32_t key, int64_t *range_sh,
-                                                 int64_t &lo, int64_t &hi) {
-  if (threadIdx.x == 0) range_sh[0] = range_sh[1] = n;
-  __syncthreads();
-  for (int64_t r = threadIdx.x; r < n; r += blockDim.x) {
-    const int32_t v = sid[r];
-    const bool first = r == 0;
-    const int32_t prev = first ? 0 : sid[r - 1];
-    if (v >= key && (first || prev < key)) range_sh[0] = r;
-    if (v > key && (first || prev <= key)) range_sh[1] = r;
-  }
-  __syncthreads();
-  lo = range_sh[0];
-  hi = range_sh[1];
-}
-
 static __global__ void __launch_bounds__(kSegThreads)
     segment_reduce_kernel(ChunkDev c, int32_t B, const float *row_ws, const float *coef, int mode,
-                          double *out) {
+                          const unsigned long long *bounds, double *out) {
   __shared__ double sh[3][kSegThreads];
-  __shared__ int64_t range_sh[2];
   const int32_t i = blockIdx.x;
   if (mode == 1 && !(coef[i] > 0.f)) return;
-  int64_t lo, hi;
-  sample_row_range(c.sid, c.n_rows, i, range_sh, lo, hi);
-  if (lo >= hi) return;
+  const unsigned long long lo_u = bounds[2 * (int64_t)i], hi_u = bounds[2 * (int64_t)i + 1];
+  if (lo_u >= hi_u) return;
+  const int64_t lo = (int64_t)lo_u, hi = (int64_t)hi_u;
   double cnt = 0.0, sk3 = 0.0, skl = 0.0;
   for (int64_t n = lo + threadIdx.x; n < hi; n += kSegThreads) {
     if (c.sid[n] != i || c.mask[n] == 0) continue;
@@ -306,8 +371,9 @@ static __global__ void __launch_bounds__(kSegThreads)
     const float4 ws = reinterpret_cast<const float4 *>(row_ws)[n];
     const double d = (double)ws.w;
     cnt += 1.0;
-    sk3 += exp(d) * d - expm1(d);  // rho log rho - (rho - 1), Eq. 10 integrand
-    skl += (double)ws.z;
+    const double rho = exp(d);
+    sk3 += rho * d - expm1(d);  // rho log rho - (rho - 1), Eq. 10 integrand
+    skl += c.kind == FOPD_LOSS_SAMPLED_KL ? rho * (double)ws.z : (double)ws.z;  // token loss of Eq. 12 in the chunk's form
   }
   sh[0][threadIdx.x] = cnt;
   sh[1][threadIdx.x] = sk3;

@@ -97,8 +97,9 @@ def step(chunks, dlogits, buf: BatchBuffers, tau, H, d_sup, p, rows=None, *, use
     optimise(chunks, dlogits, buf, p, rows, use_row_ws=use_row_ws, stream=stream)
 
 
-def to_chunk(d: dict, vocab=None) -> fb.Chunk:
-    return fb.Chunk(d["student"], d["teacher"], d["behav_logprob"], d["tokens"], d["mask"], d["sample_id"], vocab)
+def to_chunk(d: dict, vocab=None, loss_kind: int = fb.LOSS_FULL_KL) -> fb.Chunk:
+    return fb.Chunk(d["student"], d["teacher"], d["behav_logprob"], d["tokens"], d["mask"], d["sample_id"], vocab,
+                    loss_kind)
 
 
 # ---- vocabulary-sharded rows: every holder (rank) has a column range of every row ----

@@ -36,10 +36,11 @@ def host_chunk(d):
     return {k: v.detach().cpu() for k, v in d.items()}
 
 
-def gpu_run(chunks_dev, B, tau, H, d_sup=None, params=PARAMS, use_row_ws=True, vocab=None, want_rows=True):
+def gpu_run(chunks_dev, B, tau, H, d_sup=None, params=PARAMS, use_row_ws=True, vocab=None, want_rows=True,
+            loss_kind=0):
     dev = chunks_dev[0]["student"].device
     params = exact(params)
-    chunks = [pl.to_chunk(c, vocab) for c in chunks_dev]
+    chunks = [pl.to_chunk(c, vocab, loss_kind) for c in chunks_dev]
     buf = pl.BatchBuffers(B, dev)
     rows = [pl.RowOutputs.alloc(c["student"].shape[0], dev) for c in chunks_dev]
     dlogits = [torch.full_like(c["student"], float("nan")) for c in chunks_dev]
@@ -53,9 +54,10 @@ def gpu_run(chunks_dev, B, tau, H, d_sup=None, params=PARAMS, use_row_ws=True, v
     return buf, rows, dlogits, bits
 
 
-def oracle_run(chunks_host, B, tau, H, d_sup=None, params=PARAMS):
+def oracle_run(chunks_host, B, tau, H, d_sup=None, params=PARAMS, loss_kind=0):
     params = exact(params)
-    return orc.run_batch(chunks_host, B, tau, H, d_sup, params["alpha"], params["beta"], params["xi"], params["lam"])
+    return orc.run_batch(chunks_host, B, tau, H, d_sup, params["alpha"], params["beta"], params["xi"], params["lam"],
+                         loss_kind)
 
 
 def out_ulp(dtype):
@@ -118,10 +120,15 @@ def gpu_run_vocab_sharded(cuts):
 
 
 def compare(chunks_dev, B, tau, H, d_sup=None, params=PARAMS, use_row_ws=True, grad_rows_per_chunk=None,
-            seed=0, expect_bits=0, vocab=None, runner=None):
-    """Full comparison of one batch; returns a dict of the maxima seen."""
+            seed=0, expect_bits=0, vocab=None, runner=None, loss_kind=0):
+    """Full comparison of one batch; returns a dict of the maxima seen.  loss_kind 1: the
+    sampled-token form of the token loss (the oracle's per-token loss then stands in its kl field)."""
     params = exact(params)
-    buf, rows, dlogits, bits = (runner or gpu_run)(chunks_dev, B, tau, H, d_sup, params, use_row_ws, vocab)
+    if loss_kind:
+        assert runner is None
+        buf, rows, dlogits, bits = gpu_run(chunks_dev, B, tau, H, d_sup, params, use_row_ws, vocab, loss_kind=loss_kind)
+    else:
+        buf, rows, dlogits, bits = (runner or gpu_run)(chunks_dev, B, tau, H, d_sup, params, use_row_ws, vocab)
     assert bits == expect_bits, f"device status bits {bits}"
     V = vocab or chunks_dev[0]["student"].shape[1]
     hc = [host_chunk(c) for c in chunks_dev]
@@ -129,7 +136,7 @@ def compare(chunks_dev, B, tau, H, d_sup=None, params=PARAMS, use_row_ws=True, g
         for c in hc:
             c["student"] = c["student"][:, :V].contiguous()
             c["teacher"] = c["teacher"][:, :V].contiguous()
-    ref = oracle_run(hc, B, tau, H, d_sup, params)
+    ref = oracle_run(hc, B, tau, H, d_sup, params, loss_kind)
     out = dict(lp=0.0, kl=0.0, ratio=0.0, f=0.0, loss=0.0, grad_abs=0.0, grad_rel=0.0, rowsum=0.0, grad_max=0.0)
 
     # ---- per-token outputs
@@ -146,7 +153,7 @@ def compare(chunks_dev, B, tau, H, d_sup=None, params=PARAMS, use_row_ws=True, g
             out["lp"] = max(out["lp"], np.abs(g["lp_s"] - st.lp_s)[valid].max(), np.abs(g["lp_t"] - st.lp_t)[valid].max())
             if use_row_ws:
                 out["lp"] = max(out["lp"], np.abs(ws[:, 0] - st.lse_s)[valid].max(), np.abs(ws[:, 1] - st.lse_t)[valid].max())
-            out["kl"] = max(out["kl"], (np.abs(g["kl"] - st.kl) / np.maximum(1.0, st.kl))[valid].max())
+            out["kl"] = max(out["kl"], (np.abs(g["kl"] - st.kl) / np.maximum(1.0, np.abs(st.kl)))[valid].max())
             out["ratio"] = max(out["ratio"], (np.abs(g["ratio"] - st.rho)[valid] / st.rho[valid]).max())
     assert out["lp"] <= TOL_LOGPROB, out
     assert out["kl"] <= 1e-4, out
@@ -213,7 +220,7 @@ def compare(chunks_dev, B, tau, H, d_sup=None, params=PARAMS, use_row_ws=True, g
             must = np.concatenate([must, edges, edges + 1])
             sel = np.unique(np.concatenate([must, rng.choice(n, size=grad_rows_per_chunk, replace=False)]))
         g_ref = orc.grad_rows(c["student"], c["teacher"], c["tokens"], c["behav_logprob"], c["mask"],
-                              c["sample_id"], fr.coef, params["lam"], sel)
+                              c["sample_id"], fr.coef, params["lam"], sel, loss_kind)
         g_gpu = dl[torch.as_tensor(sel, device=dl.device)][:, :V].double().cpu().numpy()
         err = np.abs(g_gpu - g_ref)
         out["grad_abs"] = max(out["grad_abs"], float(err.max()))
@@ -236,6 +243,13 @@ def compare(chunks_dev, B, tau, H, d_sup=None, params=PARAMS, use_row_ws=True, g
         # d = lp_s - b carries the absolute fp32 error of the log-normaliser (~1e-6), so the
         # anchor term lambda * rho * d at the stored token has an absolute, not relative, error
         bound[np.arange(len(sel)), ycol] += 1e-5 * np.abs(cf * params["lam"] * st.rho[sel] * (1 + np.abs(st.d[sel])))
+        if loss_kind:
+            # the row is weight * (1[v = y] - p_s(v)) with weight = coef rho (r + lambda d); r and d carry
+            # the absolute fp32 error of the log-normalisers (~1e-6 each), whatever their own size
+            onehot = np.zeros_like(cp)
+            onehot[np.arange(len(sel)), ycol] = 1.0
+            p_s = np.exp(S64 - st.lse_s[sel, None])
+            bound += 1e-5 * np.abs(cf * st.rho[sel])[:, None] * np.abs(onehot - p_s)
         out["grad_rel"] = max(out["grad_rel"], float((err / bound).max()))
     # 1e-5 absolute, unless the rounding of the largest output alone exceeds it (tests with
     # a handful of rows per sample have per-token weights ~1e-2, far above any real batch)

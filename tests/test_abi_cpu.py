@@ -35,20 +35,21 @@ def test_library_exports_every_declared_symbol(lib):
 
 
 def test_strerror_covers_every_status(lib):
-    seen = {fb.strerror(c) for c in range(0, -9, -1)}
-    assert len(seen) == 9 and "unknown fopd status" not in seen
+    seen = {fb.strerror(c) for c in range(0, -10, -1)}
+    assert len(seen) == 10 and "unknown fopd status" not in seen
     assert fb.strerror(-99) == "unknown fopd status"
 
 
 def _chunk(**kw):
     base = dict(student=0x1000, teacher=0x2000, behav_logprob=0x3000, tokens=0x4000, mask=0x5000,
-                sample_id=0x6000, n_rows=4, vocab=64, row_stride=64, dtype=0)
+                sample_id=0x6000, n_rows=4, vocab=64, row_stride=64, dtype=0, loss_kind=0)
     base.update(kw)
     return fb.fopd_chunk(*[base[f] for f, _ in fb.fopd_chunk._fields_])
 
 
 @pytest.mark.parametrize("kw,code", [
     (dict(dtype=7), -4),
+    (dict(loss_kind=2), -9),
     (dict(n_rows=-1), -3),
     (dict(vocab=0), -3),
     (dict(row_stride=32), -3),

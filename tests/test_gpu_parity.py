@@ -324,6 +324,55 @@ def test_many_short_samples_and_chunk_without_aligned_rows():
     print(out)
 
 
+def test_thousands_of_samples_over_a_quarter_million_rows():
+    """4,096 samples of 64 rows each (262,144 rows, small vocabulary): the per-sample reduction
+    finds every sample's row range in one pass over the rows, so its cost does not grow with the
+    number of samples times the number of rows.  Results against the oracle; the time of the
+    statistics call with 4,096 samples against the same rows in 64 samples."""
+    rng = np.random.RandomState(11)
+    n, V = 262_144, 128
+    times = {}
+    for B in (4096, 64):
+        sid = np.repeat(np.arange(B, dtype=np.int32), n // B)
+        mask = (rng.rand(n) > 0.2).astype(np.uint8)
+        wl = synth.Workload("many", B, V, torch.bfloat16, n, sid, mask, rng.randint(0, 5, size=B).astype(np.int32),
+                            np.full(B, n // B, np.int32), seed=B)
+        chunks = _chunks(wl)
+        if B == 4096:
+            print(par.compare(chunks, B, wl.tau, wl.H, grad_rows_per_chunk=64))
+        ch = pl.to_chunk(chunks[0])
+        buf = pl.BatchBuffers(B, DEV)
+        ws = torch.empty((n, 4), dtype=torch.float32, device=DEV)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for it in range(6):
+            if it == 1:
+                e0.record()
+            fb.fopd_token_stats(ch, B, buf.acc, row_ws=ws, status=buf.status)
+        e1.record()
+        torch.cuda.synchronize()
+        times[B] = e0.elapsed_time(e1) / 5
+    print("fopd_token_stats ms per call by number of samples:", times)
+    assert times[4096] < 3.0 * times[64] + 0.1
+
+
+def test_out_of_range_sample_id_in_the_middle_of_a_sample():
+    """A bad sample id is flagged and its row treated as masked wherever it sits; the sample it
+    interrupts keeps the sums of its other rows, identically on every run."""
+    wl = synth.tool_use(scale=1 / 32)
+    chunks = _chunks(wl)
+    for c in chunks[:2]:
+        sid = c["sample_id"].clone()
+        mid = sid.numel() // 2
+        sid[mid] = -1
+        sid[mid + 3] = wl.B + 5
+        c["sample_id"] = sid
+    out = par.compare(chunks, wl.B, wl.tau, wl.H, expect_bits=2, grad_rows_per_chunk=32)
+    a = par.gpu_run(chunks, wl.B, wl.tau, wl.H)
+    b = par.gpu_run(chunks, wl.B, wl.tau, wl.H)
+    assert torch.equal(a[0].acc, b[0].acc) and torch.equal(a[0].loss, b[0].loss)
+    print(out)
+
+
 def test_two_streams_run_two_batches_concurrently():
     """Disjoint buffers on two non-default streams give the same results as one after the other."""
     wl = synth.reasoning(scale=1 / 32)

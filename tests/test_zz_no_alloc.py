@@ -83,5 +83,9 @@ def test_static_scratch_entry_rejects_oversized_chunks():
     rc = fb.lib().fopd_token_stats_static(ctypes.byref(c), wl.B, None, None, None, None,
                                           ctypes.c_void_p(buf.acc.data_ptr()), None, None)
     assert rc == -3
+    c.n_rows = 4
+    rc = fb.lib().fopd_token_stats_static(ctypes.byref(c), fb.STATIC_MAX_SAMPLES + 1, None, None, None, None,
+                                          ctypes.c_void_p(buf.acc.data_ptr()), None, None)
+    assert rc == -3  # more samples than the built-in row-range array holds
     torch.cuda.synchronize()
     assert float(buf.acc.abs().sum()) == 0.0
