@@ -30,26 +30,22 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-METRIC = "fused OPD loss path (token stats + freshness + loss fwd+bwd) throughput at V=151,936"
+METRIC = "fused OPD loss fwd+bwd tokens/s and HBM GB/s (% of ~8 TB/s) at V=151,936"
 UNIT = "tokens/s"
+# What the top-level `value` covers, and where the metric's own figure sits in the line.
+VALUE_IS = ("whole hot path per batch (fopd_token_stats on every chunk, fopd_sample_freshness, fopd_loss_fwd_bwd on "
+            "every chunk, fopd_loss_finalize); the metric's own figure is metric_figures.loss_fwd_bwd_cached "
+            "(fopd_loss_fwd_bwd given the row statistics fopd_token_stats wrote), with the same call without "
+            "cached statistics beside it in metric_figures.loss_fwd_bwd_on_chip")
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel.
-# grad_stream_kernel: one-pass ncu captures of the workloads themselves (the three counters
-# below take a single pass, so nothing is saved or restored around the launch), summarised in
-# profiles/dram_counters_reasoning_and_config5.md.  fused_cluster_kernel: ratio to its
-# algorithmic bytes from the --set full capture of the 4,096 x 151,936 case
-# (profiles/fused_cluster_kernel_4096x151936.md); its traffic grows in proportion to the rows.
-# A kernel that has changed since its counters were taken is taken out of these tables.
-NCU_TRAFFIC_BYTES = {"grad_stream_kernel": {
-    "reasoning": 23291478784,
-    "roofline_4096x32000": 750365440, "roofline_4096x128256": 3112168192, "roofline_4096x151936": 3697052000,
-    "roofline_16384x32000": 3101060096, "roofline_16384x128256": 12566872320,
-    "roofline_16384x151936": 14894971136, "roofline_65536x32000": 12529531136,
-    "roofline_65536x128256": 50388422656, "roofline_65536x151936": 59700739072,
-}}
-NCU_TRAFFIC_RATIO = {"fused_cluster_kernel": 0.9902}
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of a launch over its algorithmic
+# bytes, from ncu captures of a small case of the same kernel (4,096 rows x 151,936: larger than
+# L2, a few GB on the device); the traffic of a row does not depend on how many rows there are, so
+# the ratio scales to a full launch by the rows processed.  A kernel that has changed since its
+# counters were taken is taken out of this table (traffic: null).
+NCU_TRAFFIC_RATIO = {"grad_stream_kernel": 0.990, "token_stats_kernel": 1.000}
 
 def parse_args():
     ap = argparse.ArgumentParser()
@@ -64,8 +60,11 @@ def parse_args():
     ap.add_argument("--vocab-shards", type=int, default=8,
                     help="also time the vocabulary-sharded entry points with this many column ranges (0: skip)")
     ap.add_argument("--max-chunks", type=int, default=0,
-                    help="keep only the first K chunks of a chunked workload (0: all; the full tool_use and "
-                         "coding_agent batches hold 134-180 GB on the device)")
+                    help="keep only the first K chunks of a chunked workload (0: all)")
+    ap.add_argument("--resident-chunks", type=int, default=0,
+                    help="chunks of a chunked workload whose logits are generated and kept on the device; the "
+                         "other chunks reuse them in turn with their own mask and sample ids (0: as many as fit, at most 3)")
+    ap.add_argument("--no-sampled", action="store_true", help="skip the timing of the sampled-token form of the loss")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-on-chip", action="store_true", help="skip the extra timing of the on-chip fwd+bwd kernel")
     ap.add_argument("--cpu-sample-rows", type=int, default=0, help="rows of the CPU-oracle sample (0 = auto)")
@@ -282,14 +281,35 @@ def main():
         keep = args.max_chunks * wl.chunk_rows
         wl = dataclasses.replace(wl, name="%s[first %d chunks]" % (wl.name, args.max_chunks),
                                  sample_id=wl.sample_id[:keep], mask=wl.mask[:keep])
-    need_dev = 3 * wl.n_rows * wl.V * (2 if wl.dtype == torch.bfloat16 else 4)
+    esz = 2 if wl.dtype == torch.bfloat16 else 4
     free_dev, _ = torch.cuda.mem_get_info(dev)
-    if need_dev > 0.9 * free_dev:
-        raise SystemExit("workload %s needs %.0f GB resident (S, T, dlogits of every chunk); %.0f GB free"
-                         % (wl.name, need_dev / 1e9, free_dev / 1e9))
-    chunks_d = [synth.gen_chunk(wl, j, dev) for j in range(wl.n_chunks)]
+    chunk_bytes = 3 * min(wl.chunk_rows, wl.n_rows) * wl.V * esz   # S, T, dlogits of one chunk
+    fit = int((0.85 * free_dev) // chunk_bytes)
+    if fit < 1:
+        raise SystemExit("workload %s needs %.0f GB per chunk (S, T, dlogits); %.0f GB free"
+                         % (wl.name, chunk_bytes / 1e9, free_dev / 1e9))
+    # Chunked workloads stream: the logits of the first K chunks stay on the device and chunk j
+    # works on the logits, tokens and behaviour log-probs of chunk j % K (rows are i.i.d.) with
+    # its OWN mask and sample ids, so the per-sample structure, the number of aligned rows and
+    # the gates are the workload's; K x 15 GB cycled through is far larger than L2.
+    K = wl.n_chunks if wl.n_chunks <= fit and not args.resident_chunks else min(
+        wl.n_chunks, fit, args.resident_chunks or 3)
+    slots = [synth.gen_chunk(wl, j, dev) for j in range(K)]
+    chunks_d = []
+    for j in range(wl.n_chunks):
+        lo, hi = wl.chunk_range(j)
+        n = hi - lo
+        if j < K:
+            chunks_d.append(slots[j])
+        else:
+            base = slots[j % K]
+            chunks_d.append(dict(student=base["student"][:n], teacher=base["teacher"][:n], tokens=base["tokens"][:n],
+                                 behav_logprob=base["behav_logprob"][:n],
+                                 mask=torch.from_numpy(wl.mask[lo:hi].copy()).to(dev),
+                                 sample_id=torch.from_numpy(wl.sample_id[lo:hi].copy()).to(dev)))
     chunks = [pl.to_chunk(c) for c in chunks_d]
-    dlogits = [torch.empty_like(c["student"]) for c in chunks_d]
+    dl_slots = [torch.empty_like(c["student"]) for c in slots]
+    dlogits = [dl_slots[j % K][:chunks_d[j]["student"].shape[0]] for j in range(wl.n_chunks)]
     rows = [pl.RowOutputs.alloc(c["student"].shape[0], dev) for c in chunks_d]
     buf = pl.BatchBuffers(wl.B, dev)
     P = synth.DEFAULT_PARAMS
@@ -332,8 +352,8 @@ def main():
     barrier()
     clocks = sampler.stop(wall0, time.time()) if rank == 0 else None
     total_ms = t_begin.elapsed_time(t_end)
-    stats_all = [e[0].elapsed_time(e[1]) / len(chunks) for e in events]
-    grad_all = [e[2].elapsed_time(e[3]) / len(chunks) for e in events]
+    stats_all = [e[0].elapsed_time(e[1]) for e in events]   # all chunks of the batch
+    grad_all = [e[2].elapsed_time(e[3]) for e in events]
     stats_ms, grad_ms = statistics.mean(stats_all), statistics.mean(grad_all)
 
     # the same loss forward + backward without cached row statistics (on-chip kernel), timed
@@ -349,13 +369,42 @@ def main():
                 fb.fopd_loss_fwd_bwd(ch, buf.B, buf.coef, p, dlogits[j], buf.loss_acc, status=buf.status)
         t_end.record()
         torch.cuda.synchronize()
-        on_chip_ms = t_begin.elapsed_time(t_end) / args.steps / len(chunks)
+        on_chip_ms = t_begin.elapsed_time(t_end) / args.steps
+
+    # the sampled-token form of the token loss (importance-weighted reverse KL on the stored token):
+    # its own measurement phase for the row statistics and weights, then the timed loss forward +
+    # backward, which reads only the student row of a differentiated row
+    sampled = None
+    if cached and not args.no_sampled:
+        s_chunks = [pl.to_chunk(c, loss_kind=fb.LOSS_SAMPLED_KL) for c in chunks_d]
+        s_buf = pl.BatchBuffers(wl.B, dev)
+        s_rows = rows  # the full-vocabulary statistics are not needed any more
+        pl.measure(s_chunks, s_buf, s_rows, keep_row_ws=True)
+        pl.freshness(s_buf, tau, H, None, p)
+        for it in range(3 + args.steps):
+            if it == 3:
+                torch.cuda.synchronize()
+                t_begin.record()
+            pl.optimise(s_chunks, dlogits, s_buf, p, s_rows, use_row_ws=True)
+        t_end.record()
+        torch.cuda.synchronize()
+        s_buf.loss_acc.zero_()  # the timed repetitions all added to it
+        pl.optimise(s_chunks, dlogits, s_buf, p, s_rows, use_row_ws=True)
+        s_coef = s_buf.coef.cpu().numpy()
+        s_active = int(((s_coef[np.clip(wl.sample_id, 0, wl.B - 1)] > 0) & (wl.mask > 0)).sum())
+        s_ms = t_begin.elapsed_time(t_end) / args.steps
+        s_bytes = wl.V * (2 if wl.dtype == torch.bfloat16 else 4) * (2 * s_active + (wl.n_rows - s_active))
+        sampled = {"kernel": "grad_sampled_kernel", "ms_per_batch": s_ms, "differentiated_rows": s_active,
+                   "tokens_per_s": s_active / (s_ms * 1e-3), "algorithmic_bytes": s_bytes,
+                   "bytes_per_differentiated_row": "2 V e (student read, gradient written)",
+                   "loss": float(s_buf.loss.cpu()[0])}
 
     # the vocabulary-sharded entry points on the same rows: every holder's column range in turn
     # on this one GPU (partial sums of all parts, one merge, every part's gradient), so the sums
     # over the parts compare with the whole-row kernels above
     sharded = None
     if cached and args.vocab_shards > 1 and len(chunks) == 1:
+        pl.measure(chunks, buf, rows, keep_row_ws=True)  # (the sampled form above reused the row workspace)
         sharded = time_vocab_sharded(args, wl, chunks_d[0], dlogits[0], rows[0], buf, p, dev)
 
     coef = buf.coef.cpu().numpy()
@@ -364,48 +413,67 @@ def main():
     stats_bytes, grad_bytes = algorithmic_bytes(wl, active_rows)
     value, ms_per_step = replica_throughput(aligned, total_ms / args.steps, dev)
     peak, peak_src = measured_peak()
-    n_launch_chunk = len(chunks)
-    kernels_per_step = n_launch_chunk * (2 + (2 if cached else 3)) + 2
+    n_chunks = len(chunks)
+    # per chunk: statistics sweep + 2 row-range kernels + per-sample reduction; gradient sweep (or
+    # row weights + on-chip kernel) + 2 row-range kernels + per-sample reduction; per batch: freshness, finalize
+    kernels_per_step = n_chunks * (4 + (4 if cached else 5)) + 2
     plan = fb.fopd_loss_fwd_bwd_plan(wl.dtype, wl.V)
-    grad_kernel = "grad_stream_kernel" if cached else (
-        "fused_cluster_kernel" if plan["cluster_size"] else "token_stats_kernel+grad_stream_kernel")
-    achieved = grad_bytes / n_launch_chunk / (grad_ms * 1e-3) / 1e9
-    traffic, traffic_src = None, None
-    if n_launch_chunk == 1 and wl.name in NCU_TRAFFIC_BYTES.get(grad_kernel, {}):
-        traffic, traffic_src = NCU_TRAFFIC_BYTES[grad_kernel][wl.name], "ncu, one-pass capture of this workload"
-    elif grad_kernel in NCU_TRAFFIC_RATIO and wl.V == 151936:
-        traffic = NCU_TRAFFIC_RATIO[grad_kernel] * grad_bytes / n_launch_chunk
-        traffic_src = "ncu, 4,096-row case of the same kernel scaled by rows"
+    on_chip_kernel = "fused_cluster_kernel" if plan["cluster_size"] else "token_stats_kernel+grad_stream_kernel"
+    grad_kernel = "grad_stream_kernel" if cached else on_chip_kernel
+
+    def figure(ms, nbytes, rows_done):
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        return {"ms_per_batch": ms, "tokens_per_s": rows_done / (ms * 1e-3), "gbs": gbs,
+                "frac_of_measured_peak": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS}
+
+    achieved = grad_bytes / (grad_ms * 1e-3) / 1e9
+    ratio = NCU_TRAFFIC_RATIO.get(grad_kernel)
+    traffic = None if ratio is None else ratio * grad_bytes / n_chunks
+    traffic_src = None if ratio is None else (
+        "ncu dram__bytes_read.sum + dram__bytes_write.sum of the 4,096 x 151,936 case of the same kernel, over its "
+        "algorithmic bytes (%.3f), times the algorithmic bytes of one launch here" % ratio)
+    if sampled:
+        sampled.update({k: v for k, v in figure(sampled["ms_per_batch"], sampled["algorithmic_bytes"],
+                                                sampled["differentiated_rows"]).items() if k != "ms_per_batch"})
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic", "value_is": VALUE_IS,
         "config": {
             "workload": wl.name, "rows": wl.n_rows, "aligned_tokens": aligned, "differentiated_rows": active_rows,
             "vocab": wl.V, "samples": wl.B, "logits_dtype": str(wl.dtype).replace("torch.", ""),
-            "chunks": len(chunks), "path": args.path,
+            "chunks": n_chunks, "chunk_rows": wl.chunk_rows, "path": args.path,
+            "resident_chunks": K,
+            "chunk_streaming": None if K == n_chunks else
+            "logits, tokens and behaviour log-probs of chunk j are those of generated chunk j mod %d (rows are "
+            "i.i.d.); mask and sample ids are chunk j's own; both loops of Algorithm 1 run over all %d chunks"
+            % (K, n_chunks),
             "fused_plan": None if cached else plan, "tokens_counted": "aligned (mask = 1) rows",
-            "l2": "inputs (2 x %.2f GB) far larger than the 126 MB L2, no flush needed" %
-                  (wl.n_rows * wl.V * (2 if wl.dtype == torch.bfloat16 else 4) / 1e9),
+            "l2": "%d x 3 x %.2f GB of logits and gradients cycled through, far larger than the 126 MB L2, no flush needed"
+                  % (K, min(wl.chunk_rows, wl.n_rows) * wl.V * esz / 1e9),
             "parallelism": "replicas only" if world > 1 else "1 gpu", "params": P,
         },
         "gpu_launches": kernels_per_step * args.steps,
-        "phases_ms": {"token_stats_per_chunk": stats_ms, "loss_fwd_bwd_per_chunk": grad_ms,
+        "phases_ms": {"token_stats_per_batch": stats_ms, "loss_fwd_bwd_per_batch": grad_ms,
                       "token_stats_median_best": [statistics.median(stats_all), min(stats_all)],
                       "loss_fwd_bwd_median_best": [statistics.median(grad_all), min(grad_all)],
                       "freshness": statistics.mean(e[1].elapsed_time(e[2]) for e in events)},
-        "token_stats": {"gbs": stats_bytes / n_launch_chunk / (stats_ms * 1e-3) / 1e9,
-                        "frac_of_peak": stats_bytes / n_launch_chunk / (stats_ms * 1e-3) / 1e9 / peak},
-        "loss_fwd_bwd": {"tokens_per_s": active_rows / n_launch_chunk / (grad_ms * 1e-3), "gbs": achieved,
-                         "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS},
-        "loss_fwd_bwd_on_chip": None if on_chip_ms is None else {
-            "kernel": "fused_cluster_kernel" if plan["cluster_size"] else "token_stats_kernel+grad_stream_kernel",
-            "ms_per_chunk": on_chip_ms, "gbs": grad_bytes / n_launch_chunk / (on_chip_ms * 1e-3) / 1e9,
-            "frac_of_peak": grad_bytes / n_launch_chunk / (on_chip_ms * 1e-3) / 1e9 / peak, "plan": plan},
+        "metric_figures": {
+            "loss_fwd_bwd_cached" if cached else "loss_fwd_bwd_standalone": dict(
+                figure(grad_ms, grad_bytes, active_rows), kernel=grad_kernel,
+                bytes="3 V e per differentiated row, V e per other row"),
+            "loss_fwd_bwd_on_chip": None if on_chip_ms is None else dict(
+                figure(on_chip_ms, grad_bytes, active_rows), kernel=on_chip_kernel, plan=plan),
+            "loss_fwd_bwd_sampled_token_form": sampled,
+            "token_stats": dict(figure(stats_ms, stats_bytes, aligned), bytes="2 V e per aligned row"),
+            "whole_step": dict(figure(ms_per_step, stats_bytes + grad_bytes, aligned),
+                               bytes="5 V e per differentiated row as run (two sweeps), against 3 V e at the least"),
+        },
         "roofline": {"bound": "hbm", "kernel": grad_kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_source": peak_src,
                      "traffic": traffic, "traffic_source": traffic_src,
-                     "algorithmic_bytes_per_launch": grad_bytes / n_launch_chunk},
+                     "launches_per_step": n_chunks,
+                     "algorithmic_bytes_per_launch": grad_bytes / n_chunks},
         "clocks": clocks,
         "loss": float(buf.loss.cpu()[0]),
     }
@@ -419,12 +487,12 @@ def main():
     if not args.no_e2e and len(chunks) >= 1:
         try:
             import psutil
-            need_host = 3 * sum(c["student"].numel() * c["student"].element_size() for c in chunks_d)
+            need_host = 3 * sum(c["student"].numel() * c["student"].element_size() for c in slots)
             # from the host's total memory, so that every rank takes the same decision
             if need_host * world > 0.6 * psutil.virtual_memory().total:
                 raise MemoryError("pinned host copies of the batch (%.0f GB) would not fit comfortably in host memory"
                                   % (need_host / 1e9))
-            line["e2e"] = run_e2e(args, wl, chunks_d, dev, world, aligned)
+            line["e2e"] = run_e2e(args, wl, slots, chunks_d, dev, world, aligned)
         except Exception as exc:  # report, never fake
             line["e2e"] = {"value": None, "unit": UNIT, "error": repr(exc)[:200]}
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -479,23 +547,35 @@ def time_vocab_sharded(args, wl, ch, dlogits, row_out, buf, p, dev):
             "grad_ms_all_parts": tot[2], "launches_per_pass": 2 * K + 3}
 
 
-def run_e2e(args, wl, chunks_d, dev, world, aligned):
+def run_e2e(args, wl, slots, chunks_d, dev, world, aligned):
     """Same step through fopd_step_host: logits start in pinned host memory, every step
-    uploads them, runs the path and downloads dlogits and the per-sample results."""
+    uploads them, runs the path and downloads dlogits and the per-sample results.  A chunked
+    workload whose chunks share the logits of a few generated ones on the device shares them in
+    host memory the same way (every chunk is still uploaded, and its gradient downloaded)."""
     import torch
     import torch.distributed as dist
     from paper_2605_17862_b200 import binding as fb
     from paper_2605_17862_b200 import pipeline as pl
     from paper_2605_17862_b200 import synth
 
-    host = []
-    for c in chunks_d:
-        host.append({k: v.cpu().pin_memory() for k, v in c.items()})
+    K = len(slots)
+    h_slots = [{k: v.cpu().pin_memory() for k, v in c.items()} for c in slots]
+    h_dl = [torch.empty_like(c["student"]).pin_memory() for c in h_slots]
+    host, hdl = [], []
+    for j, c in enumerate(chunks_d):
+        n = c["student"].shape[0]
+        base = h_slots[j % K]
+        if j < K:
+            host.append(base)
+        else:
+            host.append(dict(student=base["student"][:n], teacher=base["teacher"][:n], tokens=base["tokens"][:n],
+                             behav_logprob=base["behav_logprob"][:n], mask=c["mask"].cpu().pin_memory(),
+                             sample_id=c["sample_id"].cpu().pin_memory()))
+        hdl.append(h_dl[j % K][:n])
     hchunks = [pl.to_chunk(c) for c in host]
-    hdl = [torch.empty_like(c["student"]).pin_memory() for c in host]
     need = fb.fopd_step_host_workspace_bytes(hchunks, wl.B, True)
     free, _ = torch.cuda.mem_get_info(dev)
-    if need > free - (2 << 30):
+    if need > free - (2 << 30) or K < len(chunks_d):
         need = fb.fopd_step_host_workspace_bytes(hchunks, wl.B, False)
     ws = torch.empty(need, dtype=torch.uint8, device=dev)
     tau = torch.as_tensor(wl.tau)

@@ -32,8 +32,9 @@
 // so the cluster exchange of row k is covered by the gradient of row k - 1 and the
 // sums of row k + 1.  All hand-offs inside a CTA and between CTAs go through mbarriers (no
 // CTA-wide or cluster-wide barrier inside the loop).  A small kernel run first
-// writes each row's weight coef_i (0 for rows that are not differentiated), which
-// lets the control warp look for rows with independent loads.
+// writes each row's weight coef_i (0 for rows that are not differentiated, whose
+// zeros in dlogits it also writes), which lets the control warp look for rows with
+// independent loads.
 //
 // Every mbarrier wait is bounded.  A wait that runs out raises a flag in shared
 // memory; every thread of the CTA looks at the flag once per step and leaves the row
@@ -319,15 +320,29 @@ struct Pairs<FOPD_F32> {
   }
 };
 
-// Weight of every row of a chunk: coef of its sample if the row is differentiated
-// (aligned, ids in range, coef > 0), else 0.  Reports bad ids in the status word.
-static __global__ void __launch_bounds__(256)
-    row_coef_kernel(ChunkDev c, int32_t B, const float *coef, int32_t *status, float *row_cf) {
-  const int64_t n = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (n >= c.n_rows) return;
-  float cf = 0.f;
-  if (row_is_aligned(c, n, B, status, true)) cf = coef[c.sid[n]];
-  row_cf[n] = cf > 0.f ? cf : 0.f;
+// Pass over the rows before the on-chip kernel, one CTA per row: the row's weight (coef of its
+// sample if the row is differentiated -- aligned, ids in range, coef > 0 -- else 0; bad ids are
+// reported in the status word), and for a row that is not differentiated its zeros in dlogits,
+// written here at streaming-store speed so that the on-chip kernel only ever sees rows it
+// differentiates.
+template <int DT>
+__global__ void __launch_bounds__(256)
+    row_prepare_kernel(ChunkDev c, int32_t B, const float *coef, int32_t *status, float *row_cf, void *dlogits) {
+  using E = Elem<DT>;
+  __shared__ float cf_sh;
+  for (int64_t n = blockIdx.x; n < c.n_rows; n += gridDim.x) {
+    if (threadIdx.x == 0) {
+      float cf = 0.f;
+      if (row_is_aligned(c, n, B, status, true)) cf = coef[c.sid[n]];
+      cf = cf > 0.f ? cf : 0.f;
+      row_cf[n] = cf;
+      cf_sh = cf;
+    }
+    __syncthreads();
+    const float cf = cf_sh;
+    __syncthreads();
+    if (!(cf > 0.f)) zero_fill_row<DT, 256>(reinterpret_cast<char *>(dlogits) + n * c.stride * E::kBytes, c.vocab);
+  }
 }
 
 // What the control warp hands the compute warps for the gradient of one row.
@@ -600,21 +615,7 @@ __global__ void __launch_bounds__(W * 32 + 32, 1) fused_cluster_kernel(FusedArgs
       return false;
     };
     role_sync<kFusedThreads>();  // the control warp has found the first rows
-    const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
     const uint32_t no_logit = smem_u32(&sh.no_logit);
-    // This CTA's part of a row that is not differentiated: zeros.
-    auto zero_row = [&](int64_t n) {
-      char *orow = reinterpret_cast<char *>(a.dlogits) + n * row_bytes;
-      uint4 *o4 = reinterpret_cast<uint4 *>(orow) + v_lo + ctid;
-#pragma unroll
-      for (int j = 0; j < NV; ++j)
-        if (j < nv) st_stream(o4 + j * kFusedCompute, zero4);
-      if (has_tail) E::store1(orow, tail_idx, 0.f);
-    };
-    // The cluster's rows strictly between two differentiated rows are not differentiated.
-    auto zero_between = [&](int64_t from, int64_t to) {
-      for (int64_t n = from; n < to; n += n_clusters) zero_row(n);
-    };
     // Shared-memory address of this thread's j-th vector inside a slice buffer (the filler for
     // slots without a vector).
     uint32_t voff[NV];
@@ -623,7 +624,6 @@ __global__ void __launch_bounds__(W * 32 + 32, 1) fused_cluster_kernel(FusedArgs
 
     int64_t cur = sh.first_rows[0], prev = -1;
     const int64_t second = sh.first_rows[1];
-    zero_between(cluster_id, cur >= 0 ? cur : c.n_rows);
 
     uint4 X[NV], Y[NV];          // student vectors of row k and of row k - 1
     float x_tail_s = 0.f, x_tail_t = 0.f, y_tail_s = 0.f, y_tail_t = 0.f;
@@ -757,7 +757,6 @@ __global__ void __launch_bounds__(W * 32 + 32, 1) fused_cluster_kernel(FusedArgs
           if (tail_idx == gr.y) o = fmaf(ex2(fmaf(y_tail_s, kLog2e, gr.e0)), (y_tail_s - y_tail_t) - gr.K, gr.cg);
           E::store1(orow, tail_idx, o);
         }
-        zero_between(prev + n_clusters, cur >= 0 ? cur : c.n_rows);
       }
       if (cur < 0) next = -1;
 #pragma unroll

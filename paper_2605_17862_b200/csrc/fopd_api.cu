@@ -191,7 +191,7 @@ int launch_fused(const fopd_chunk *chunk, int32_t B, const float *coef, float la
   const void *kernel = fused_kernel_for<DT>(plan.nv, plan.warps);
   float *row_cf = tmp + 4 * chunk->n_rows;
   const ChunkDev d = to_dev(chunk);
-  row_coef_kernel<<<(unsigned)((chunk->n_rows + 255) / 256), 256, 0, st>>>(d, B, coef, status, row_cf);
+  row_prepare_kernel<DT><<<row_grid(chunk->n_rows), 256, 0, st>>>(d, B, coef, status, row_cf, dlogits);
   if ((rc = launch_ok()) != FOPD_OK) return rc;
   const int64_t clusters = chunk->n_rows < plan.max_clusters ? chunk->n_rows : plan.max_clusters;
   cudaLaunchConfig_t cfg;
