@@ -230,6 +230,24 @@ __device__ __forceinline__ RowAcc warp_reduce_two_step(RowAcc a) {
   return a;
 }
 
+// The same for lanes that already share their maxima: the sums add up as they are.
+__device__ __forceinline__ RowAcc warp_sum_common_scale(RowAcc a) {
+  const bool odd = threadIdx.x & 1;
+  const float give = odd ? a.zs : a.as, keep = odd ? a.as : a.zs;  // even lanes collect zs, odd lanes as
+  float za = keep + __shfl_xor_sync(0xffffffffu, give, 1);
+  float zt = a.zt + __shfl_xor_sync(0xffffffffu, a.zt, 1);
+#pragma unroll
+  for (int off = 2; off < 32; off <<= 1) {
+    za += __shfl_xor_sync(0xffffffffu, za, off);
+    zt += __shfl_xor_sync(0xffffffffu, zt, off);
+  }
+  const float other = __shfl_xor_sync(0xffffffffu, za, 1);
+  a.zs = odd ? other : za;
+  a.as = odd ? za : other;
+  a.zt = zt;
+  return a;
+}
+
 // Largest logit of a 16-byte vector.  bf16: on the packed pairs (three packed maxima), then
 // the two halves of the last pair.
 template <int DT>
@@ -657,8 +675,13 @@ __global__ void __launch_bounds__(W * 32 + 32, 1) fused_cluster_kernel(FusedArgs
           acc.ms = fmaxf(acc.ms, x_tail_s);
           acc.mt = fmaxf(acc.mt, x_tail_t);
         }
-        // the student slice is in registers now (the maximum has looked at all of it): its buffer goes back
-        __syncwarp();
+        // The warp agrees on its maxima before the exponentials, so that its lanes' sums are on one
+        // scale and merge by plain additions: the chain of dependent steps after the sweep, which
+        // all warps would sit through at the same time, shrinks to the shuffles.
+        acc.ms = warp_max(acc.ms);
+        acc.mt = warp_max(acc.mt);
+        // the student slice is in registers now (the maxima have looked at all of it): its buffer
+        // goes back (the warp-wide maximum has also brought the lanes together)
         if (lane == 0) mbar_arrive_after(smem_u32(&sh.free_s_bar[sb]), acc.ms);
         {
           const f32x2 ms2 = pack2(acc.ms, acc.ms), mt2 = pack2(acc.mt, acc.mt), l2 = pack2(kLog2e, kLog2e);
@@ -691,7 +714,7 @@ __global__ void __launch_bounds__(W * 32 + 32, 1) fused_cluster_kernel(FusedArgs
           acc.as = fmaf(e, x_tail_s - x_tail_t, acc.as);
           acc.zt += ex2((x_tail_t - acc.mt) * kLog2e);
         }
-        acc = warp_reduce_two_step(acc);
+        acc = warp_sum_common_scale(acc);
         if (lane == 0) {
           sh.warp_scratch[slot][ctid >> 5] = acc;
           mbar_arrive(smem_u32(&sh.red_bar[slot]));
