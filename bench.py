@@ -414,9 +414,10 @@ def main():
     value, ms_per_step = replica_throughput(aligned, total_ms / args.steps, dev)
     peak, peak_src = measured_peak()
     n_chunks = len(chunks)
-    # per chunk: statistics sweep + 2 row-range kernels + per-sample reduction; gradient sweep (or
-    # row weights + on-chip kernel) + 2 row-range kernels + per-sample reduction; per batch: freshness, finalize
-    kernels_per_step = n_chunks * (4 + (4 if cached else 5)) + 2
+    # per chunk: statistics sweep (+ 2 row-range kernels) + per-sample reduction; gradient sweep (or
+    # row weights + on-chip kernel) (+ 2 row-range kernels) + per-sample reduction; per batch: freshness, finalize
+    ranges = 0 if wl.B <= 32 else 2  # (batches of few samples: the reductions find the row ranges themselves)
+    kernels_per_step = n_chunks * ((2 + ranges) + ((2 if cached else 3) + ranges)) + 2
     plan = fb.fopd_loss_fwd_bwd_plan(wl.dtype, wl.V)
     on_chip_kernel = "fused_cluster_kernel" if plan["cluster_size"] else "token_stats_kernel+grad_stream_kernel"
     grad_kernel = "grad_stream_kernel" if cached else on_chip_kernel

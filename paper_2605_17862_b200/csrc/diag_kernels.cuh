@@ -140,8 +140,15 @@ static __global__ void __launch_bounds__(kSegThreads)
     divergence_reduce_kernel(const int32_t *sid, const uint8_t *mask, int64_t n_rows, const float2 *vals,
                              const unsigned long long *bounds, double *out) {
   __shared__ double sh[3][kSegThreads];
+  __shared__ unsigned long long range_sh[2];
   const int32_t i = blockIdx.x;
-  const unsigned long long lo_u = bounds[2 * (int64_t)i], hi_u = bounds[2 * (int64_t)i + 1];
+  unsigned long long lo_u, hi_u;
+  if (bounds) {
+    lo_u = bounds[2 * (int64_t)i];
+    hi_u = bounds[2 * (int64_t)i + 1];
+  } else {
+    sample_row_range(sid, n_rows, i, range_sh, lo_u, hi_u);
+  }
   if (lo_u >= hi_u) return;
   const int64_t lo = (int64_t)lo_u, hi = (int64_t)hi_u;
   double cnt = 0.0, skl = 0.0, sen = 0.0;

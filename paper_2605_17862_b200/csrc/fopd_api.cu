@@ -259,7 +259,7 @@ int fopd_token_stats(const fopd_chunk *chunk, int32_t B, float *lp_s, float *lp_
   rc = launch_stats(chunk, B, lp_s, lp_t, kl, ratio, ws, status, st);
   if (rc == FOPD_OK) rc = launch_sample_bounds(chunk->sample_id, chunk->n_rows, B, bounds, st);
   if (rc == FOPD_OK) {
-    segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(to_dev(chunk), B, ws, nullptr, 0, bounds, acc);
+    segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(to_dev(chunk), B, ws, nullptr, 0, bounds_or_null(bounds, B), acc);
     rc = launch_ok();
   }
   if (cudaFreeAsync(tmp, st) != cudaSuccess) rc = FOPD_ERR_CUDA;
@@ -324,26 +324,26 @@ int fopd_loss_fwd_bwd(const fopd_chunk *chunk, int32_t B, const float *coef, con
   if (rc == FOPD_OK && !grad_done) {
     const unsigned grid = row_grid(chunk->n_rows);
     const bool short_row = chunk->vocab / (chunk->dtype == FOPD_BF16 ? 8 : 4) < kShortRowVecs;
-#define FOPD_LAUNCH_GRAD(DT, T)                                                          \
+#define FOPD_LAUNCH_GRAD(DT, T, TS)                                                      \
   do {                                                                                     \
     if (chunk->loss_kind == FOPD_LOSS_SAMPLED_KL)                                          \
-      grad_sampled_kernel<DT, T><<<grid, T, 0, st>>>(d, B, coef, ws, p.lambda, dlogits);   \
+      grad_sampled_kernel<DT, TS><<<grid, TS, 0, st>>>(d, B, coef, ws, p.lambda, dlogits); \
     else                                                                                   \
       grad_stream_kernel<DT, T><<<grid, T, 0, st>>>(d, B, coef, ws, p.lambda, dlogits);    \
   } while (0)
     if (chunk->dtype == FOPD_BF16) {
-      if (short_row) FOPD_LAUNCH_GRAD(FOPD_BF16, kGradThreadsShortRow);
-      else FOPD_LAUNCH_GRAD(FOPD_BF16, kGradThreads);
+      if (short_row) FOPD_LAUNCH_GRAD(FOPD_BF16, kGradThreadsShortRow, kSampledThreadsShortRow);
+      else FOPD_LAUNCH_GRAD(FOPD_BF16, kGradThreads, kSampledThreads);
     } else {
-      if (short_row) FOPD_LAUNCH_GRAD(FOPD_F32, kGradThreadsShortRow);
-      else FOPD_LAUNCH_GRAD(FOPD_F32, kGradThreads);
+      if (short_row) FOPD_LAUNCH_GRAD(FOPD_F32, kGradThreadsShortRow, kSampledThreadsShortRow);
+      else FOPD_LAUNCH_GRAD(FOPD_F32, kGradThreads, kSampledThreads);
     }
 #undef FOPD_LAUNCH_GRAD
     rc = launch_ok();
   }
   if (rc == FOPD_OK) rc = launch_sample_bounds(chunk->sample_id, chunk->n_rows, B, bounds, st);
   if (rc == FOPD_OK) {
-    segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(d, B, ws, coef, 1, bounds, loss_acc);
+    segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(d, B, ws, coef, 1, bounds_or_null(bounds, B), loss_acc);
     rc = launch_ok();
   }
   if (cudaFreeAsync(blk, st) != cudaSuccess) rc = FOPD_ERR_CUDA;

@@ -35,7 +35,7 @@ int fopd_row_divergence(const void *first, const void *second, const uint8_t *ma
   rc = launch_ok();
   if (rc == FOPD_OK) rc = launch_sample_bounds(sample_id, n_rows, B, bounds, st);
   if (rc == FOPD_OK) {
-    divergence_reduce_kernel<<<B, kSegThreads, 0, st>>>(sample_id, mask, n_rows, vals, bounds, acc);
+    divergence_reduce_kernel<<<B, kSegThreads, 0, st>>>(sample_id, mask, n_rows, vals, bounds_or_null(bounds, B), acc);
     rc = launch_ok();
   }
   if (cudaFreeAsync(tmp, st) != cudaSuccess) rc = FOPD_ERR_CUDA;

@@ -67,6 +67,6 @@ extern "C" int fopd_token_stats_static(const fopd_chunk *chunk, int32_t B, float
   rc = launch_stats(chunk, B, lp_s, lp_t, kl, ratio, ws, status, st);
   if (rc != FOPD_OK) return rc;
   if ((rc = launch_sample_bounds(chunk->sample_id, chunk->n_rows, B, bounds, st)) != FOPD_OK) return rc;
-  segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(to_dev(chunk), B, ws, nullptr, 0, bounds, acc);
+  segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(to_dev(chunk), B, ws, nullptr, 0, bounds_or_null(bounds, B), acc);
   return launch_ok();
 }

@@ -103,11 +103,17 @@ static inline int scratch_release() {
 // Enqueues the pass that finds every sample's row range in a chunk (bounds: [B, 2] 64-bit).
 static inline int launch_sample_bounds(const int32_t *sid, int64_t n_rows, int32_t B, unsigned long long *bounds,
                                        cudaStream_t st) {
+  if (B <= kFewSamples) return FOPD_OK;  // the reductions find the ranges themselves (see bounds_or_null)
   sample_bounds_init_kernel<<<(unsigned)((B + 255) / 256), 256, 0, st>>>(B, bounds);
   if (n_rows > 0) sample_bounds_kernel<<<(unsigned)((n_rows + 255) / 256), 256, 0, st>>>(sid, n_rows, B, bounds);
   return launch_ok();
 }
 static inline size_t bounds_bytes(int32_t B) { return (size_t)B * 2 * sizeof(unsigned long long); }
+// What the reduction kernels are handed: the ranges launch_sample_bounds filled in, or NULL for a
+// batch of few samples, whose reduction blocks scan the ids themselves.
+static inline const unsigned long long *bounds_or_null(const unsigned long long *bounds, int32_t B) {
+  return B <= kFewSamples ? nullptr : bounds;
+}
 
 // The per-sample reduction of a chunk's row statistics with its row ranges in a temporary of
 // the library's pool.  mode 0: acc[B,4] +=; mode 1: loss_acc[B,2] += (see segment_reduce_kernel).
@@ -118,7 +124,7 @@ static inline int launch_segment_reduce(const ChunkDev &d, int32_t B, const floa
   if (rc != FOPD_OK) return rc;
   rc = launch_sample_bounds(d.sid, d.n_rows, B, bounds, st);
   if (rc == FOPD_OK) {
-    segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(d, B, row_ws, coef, mode, bounds, out);
+    segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(d, B, row_ws, coef, mode, bounds_or_null(bounds, B), out);
     rc = launch_ok();
   }
   if (cudaFreeAsync(bounds, st) != cudaSuccess) rc = FOPD_ERR_CUDA;

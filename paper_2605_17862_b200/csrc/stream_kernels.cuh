@@ -13,10 +13,13 @@
 namespace fopd {
 
 // Block sizes by row length (measured): the statistics sweep, bound by the special-function
-// pipe, wants many small CTAs per SM; the gradient sweep, bound by memory, one or two large ones.
-// Short rows take the smaller block so that more CTAs overlap their start-up.
+// pipe, wants many small CTAs per SM; the gradient sweep, bound by memory, one large one for long
+// rows.  Short rows take small blocks so that more CTAs overlap their start-up (bf16 rows of
+// 32,000: gradient sweep 6.4-6.8 TB/s with 256 threads against 6.3-6.4 with 512).
 constexpr int kStatsThreads = 256, kStatsThreadsShortRow = 128;
-constexpr int kGradThreads = 1024, kGradThreadsShortRow = 512;
+constexpr int kGradThreads = 1024, kGradThreadsShortRow = 256;
+// the sampled-token gradient sweep (one read, one write per element) wants more CTAs per SM in flight
+constexpr int kSampledThreads = 512, kSampledThreadsShortRow = 256;
 constexpr int64_t kShortRowVecs = 8192;  // rows of fewer 16-byte vectors count as short
 constexpr int kUnroll = 4;
 constexpr int64_t kMaxGrid = 1 << 30;
@@ -347,8 +350,31 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads)
   }
 }
 
+// The same range for one sample, found by the block that reduces it (all threads scan the
+// chunk's ids together; shared-memory minimum / maximum over the runs).  Costs a pass over the
+// ids per sample, which is what a batch of a few samples wants: no extra launches.
+constexpr int32_t kFewSamples = 32;
+__device__ __forceinline__ void sample_row_range(const int32_t *sid, int64_t n_rows, int32_t key,
+                                                 unsigned long long *range_sh, unsigned long long &lo,
+                                                 unsigned long long &hi) {
+  if (threadIdx.x == 0) {
+    range_sh[0] = ~0ull;
+    range_sh[1] = 0ull;
+  }
+  __syncthreads();
+  for (int64_t n = threadIdx.x; n < n_rows; n += blockDim.x) {
+    if (sid[n] != key) continue;
+    if (n == 0 || sid[n - 1] != key) atomicMin(&range_sh[0], (unsigned long long)n);
+    if (n == n_rows - 1 || sid[n + 1] != key) atomicMax(&range_sh[1], (unsigned long long)(n + 1));
+  }
+  __syncthreads();
+  lo = range_sh[0];
+  hi = range_sh[1];
+}
+
 // a5: deterministic segmented reduction of per-row statistics into per-sample
-// sums.  One block per sample over the sample's row range; every thread sums a
+// sums.  One block per sample over the sample's row range (from `bounds`, or found here when
+// bounds is NULL); every thread sums a
 // fixed strided subset in fp64 and a fixed tree combines them, so a rerun
 // reproduces the bits.  mode 0: acc[B,4] += {cnt, sum k3, sum kl, rows}.
 // mode 1: loss_acc[B,2] += {sum kl, sum k3} over rows of samples with coef > 0.
@@ -358,9 +384,16 @@ static __global__ void __launch_bounds__(kSegThreads)
     segment_reduce_kernel(ChunkDev c, int32_t B, const float *row_ws, const float *coef, int mode,
                           const unsigned long long *bounds, double *out) {
   __shared__ double sh[3][kSegThreads];
+  __shared__ unsigned long long range_sh[2];
   const int32_t i = blockIdx.x;
   if (mode == 1 && !(coef[i] > 0.f)) return;
-  const unsigned long long lo_u = bounds[2 * (int64_t)i], hi_u = bounds[2 * (int64_t)i + 1];
+  unsigned long long lo_u, hi_u;
+  if (bounds) {
+    lo_u = bounds[2 * (int64_t)i];
+    hi_u = bounds[2 * (int64_t)i + 1];
+  } else {
+    sample_row_range(c.sid, c.n_rows, i, range_sh, lo_u, hi_u);
+  }
   if (lo_u >= hi_u) return;
   const int64_t lo = (int64_t)lo_u, hi = (int64_t)hi_u;
   double cnt = 0.0, sk3 = 0.0, skl = 0.0;

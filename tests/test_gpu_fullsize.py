@@ -249,13 +249,15 @@ def test_reasoning_full_size_from_host_buffers():
         assert bool(torch.isfinite(dl[j]).all()), "a gradient row was never written"
 
 
-@pytest.mark.parametrize("name,use_row_ws", [("tool_use", True), ("coding_agent", False)])
+@pytest.mark.parametrize("name,use_row_ws", [("tool_use", True), ("tool_use", False), ("coding_agent", False),
+                                             ("coding_agent", True)])
 def test_chunked_workloads_full_size(name, use_row_ws):
     wl = synth.WORKLOADS[name]()  # 16,384-row chunks cutting across samples, V = 151,936
     print(wl.name, wl.n_rows, wl.V, wl.n_chunks, _run_full_size(wl, use_row_ws))
 
 
-@pytest.mark.parametrize("rows,V,use_row_ws", [(4096, 32000, False), (16384, 128256, True), (65536, 151936, False)])
+@pytest.mark.parametrize("rows,V,use_row_ws", [(4096, 32000, False), (16384, 128256, True), (65536, 151936, False),
+                                               (4096, 151936, False), (65536, 32000, True), (16384, 151936, True)])
 def test_roofline_points_full_size(rows, V, use_row_ws):
     wl = synth.roofline_point(rows, V)
     print(wl.name, _run_full_size(wl, use_row_ws))
