@@ -32,9 +32,9 @@
 // so the cluster exchange of row k is covered by the gradient of row k - 1 and the
 // sums of row k + 1.  All hand-offs inside a CTA and between CTAs go through mbarriers (no
 // CTA-wide or cluster-wide barrier inside the loop).  A small kernel run first
-// writes each row's weight coef_i (0 for rows that are not differentiated, whose
-// zeros in dlogits it also writes), which lets the control warp look for rows with
-// independent loads.
+// writes each row's weight coef_i (0 for rows that are not differentiated), which
+// lets the control warp look for rows with independent loads; the zeros of those
+// rows are written by a kernel that runs beside this one.
 //
 // Every mbarrier wait is bounded.  A wait that runs out raises a flag in shared
 // memory; every thread of the CTA looks at the flag once per step and leaves the row
@@ -338,29 +338,32 @@ struct Pairs<FOPD_F32> {
   }
 };
 
-// Pass over the rows before the on-chip kernel, one CTA per row: the row's weight (coef of its
-// sample if the row is differentiated -- aligned, ids in range, coef > 0 -- else 0; bad ids are
-// reported in the status word), and for a row that is not differentiated its zeros in dlogits,
-// written here at streaming-store speed so that the on-chip kernel only ever sees rows it
-// differentiates.
+// Weight of every row of a chunk, written before the on-chip kernel: coef of its sample if the
+// row is differentiated (aligned, ids in range, coef > 0), else 0.  Reports bad ids in the
+// status word.
+static __global__ void __launch_bounds__(256)
+    row_weight_kernel(ChunkDev c, int32_t B, const float *coef, int32_t *status, float *row_cf) {
+  const int64_t n = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (n >= c.n_rows) return;
+  float cf = 0.f;
+  if (row_is_aligned(c, n, B, status, true)) cf = coef[c.sid[n]];
+  row_cf[n] = cf > 0.f ? cf : 0.f;
+}
+
+// Zeros for the rows the on-chip kernel does not differentiate, one CTA per row, so that the
+// on-chip kernel only ever sees rows it works on.  Launched AFTER the on-chip kernel with
+// programmatic stream serialisation: the on-chip kernel lets its dependents go at once, so
+// these CTAs run next to it on the SMs its clusters leave free (13 of 148 with clusters of
+// nine) and, whatever is left when it ends, on all SMs.  The two kernels write disjoint rows.
+// CTA 0 ends by waiting for the on-chip kernel, so that this grid -- which is what the next
+// launch in the stream waits for -- is not complete before the on-chip kernel is.
 template <int DT>
-__global__ void __launch_bounds__(256)
-    row_prepare_kernel(ChunkDev c, int32_t B, const float *coef, int32_t *status, float *row_cf, void *dlogits) {
+__global__ void __launch_bounds__(256) zero_rows_kernel(ChunkDev c, const float *row_cf, void *dlogits) {
   using E = Elem<DT>;
-  __shared__ float cf_sh;
-  for (int64_t n = blockIdx.x; n < c.n_rows; n += gridDim.x) {
-    if (threadIdx.x == 0) {
-      float cf = 0.f;
-      if (row_is_aligned(c, n, B, status, true)) cf = coef[c.sid[n]];
-      cf = cf > 0.f ? cf : 0.f;
-      row_cf[n] = cf;
-      cf_sh = cf;
-    }
-    __syncthreads();
-    const float cf = cf_sh;
-    __syncthreads();
-    if (!(cf > 0.f)) zero_fill_row<DT, 256>(reinterpret_cast<char *>(dlogits) + n * c.stride * E::kBytes, c.vocab);
-  }
+  for (int64_t n = blockIdx.x; n < c.n_rows; n += gridDim.x)
+    if (!(row_cf[n] > 0.f))
+      zero_fill_row<DT, 256>(reinterpret_cast<char *>(dlogits) + n * c.stride * E::kBytes, c.vocab);
+  if (blockIdx.x == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // What the control warp hands the compute warps for the gradient of one row.
@@ -434,6 +437,8 @@ __global__ void __launch_bounds__(W * 32 + 32, 1) fused_cluster_kernel(FusedArgs
   const bool has_tail = owns_tail && !control && tail_idx < V;
   const int64_t row_bytes = c.stride * E::kBytes;
 
+  // the kernel that writes the zeros of the other rows may start now (it needs nothing from here)
+  asm volatile("griddepcontrol.launch_dependents;");
   if (tid == 0) {
     for (int b = 0; b < kStudentBufs; ++b) {
       mbar_init(smem_u32(&sh.load_s_bar[b]), 1);

@@ -191,7 +191,7 @@ int launch_fused(const fopd_chunk *chunk, int32_t B, const float *coef, float la
   const void *kernel = fused_kernel_for<DT>(plan.nv, plan.warps);
   float *row_cf = tmp + 4 * chunk->n_rows;
   const ChunkDev d = to_dev(chunk);
-  row_prepare_kernel<DT><<<row_grid(chunk->n_rows), 256, 0, st>>>(d, B, coef, status, row_cf, dlogits);
+  row_weight_kernel<<<(unsigned)((chunk->n_rows + 255) / 256), 256, 0, st>>>(d, B, coef, status, row_cf);
   if ((rc = launch_ok()) != FOPD_OK) return rc;
   const int64_t clusters = chunk->n_rows < plan.max_clusters ? chunk->n_rows : plan.max_clusters;
   cudaLaunchConfig_t cfg;
@@ -209,9 +209,26 @@ int launch_fused(const fopd_chunk *chunk, int32_t B, const float *coef, float la
   void *args[] = {&a};
   // the attributes are per function, and the plan of another vocabulary may have changed them:
   // set them and launch under one lock, so that a call from another thread cannot come between
-  std::lock_guard<std::mutex> lock(g_fused_mu);
-  if ((rc = set_fused_attributes(kernel, C, plan.smem)) != FOPD_OK) return rc;
-  if (cudaLaunchKernelExC(&cfg, kernel, args) != cudaSuccess) {
+  {
+    std::lock_guard<std::mutex> lock(g_fused_mu);
+    if ((rc = set_fused_attributes(kernel, C, plan.smem)) != FOPD_OK) return rc;
+    if (cudaLaunchKernelExC(&cfg, kernel, args) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return FOPD_ERR_CUDA;
+    }
+  }
+  // the zeros of the rows that are not differentiated, beside the on-chip kernel (see zero_rows_kernel)
+  cudaLaunchAttribute zattr[1];
+  zattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  zattr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t zcfg = cudaLaunchConfig_t{};
+  zcfg.blockDim = dim3(256);
+  zcfg.gridDim = dim3(row_grid(chunk->n_rows));
+  zcfg.stream = st;
+  zcfg.attrs = zattr;
+  zcfg.numAttrs = 1;
+  const float *row_cf_c = row_cf;
+  if (cudaLaunchKernelEx(&zcfg, zero_rows_kernel<DT>, d, row_cf_c, dlogits) != cudaSuccess) {
     (void)cudaGetLastError();
     return FOPD_ERR_CUDA;
   }
