@@ -248,18 +248,29 @@ __device__ __forceinline__ RowAcc warp_sum_common_scale(RowAcc a) {
   return a;
 }
 
-// Largest logit of a 16-byte vector.  bf16: on the packed pairs (three packed maxima), then
-// the two halves of the last pair.
-template <int DT>
-__device__ __forceinline__ float vec_max(const uint4 &v) {
+// Largest logit of N 16-byte vectors.  bf16: packed maxima over all words first, then the two
+// halves of the one word that is left.
+template <int DT, int N>
+__device__ __forceinline__ float vecs_max(const uint4 (&v)[N]) {
   if (DT == FOPD_BF16) {
-    __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162 *>(&v.x), b = *reinterpret_cast<const __nv_bfloat162 *>(&v.y),
-                   c = *reinterpret_cast<const __nv_bfloat162 *>(&v.z), d = *reinterpret_cast<const __nv_bfloat162 *>(&v.w);
-    const __nv_bfloat162 m = __hmax2(__hmax2(a, b), __hmax2(c, d));
+    __nv_bfloat162 m;
+#pragma unroll
+    for (int j = 0; j < N; ++j) {
+      const __nv_bfloat162 a = *reinterpret_cast<const __nv_bfloat162 *>(&v[j].x),
+                           b = *reinterpret_cast<const __nv_bfloat162 *>(&v[j].y),
+                           c = *reinterpret_cast<const __nv_bfloat162 *>(&v[j].z),
+                           d = *reinterpret_cast<const __nv_bfloat162 *>(&v[j].w);
+      const __nv_bfloat162 mj = __hmax2(__hmax2(a, b), __hmax2(c, d));
+      m = j == 0 ? mj : __hmax2(m, mj);
+    }
     const uint32_t w = *reinterpret_cast<const uint32_t *>(&m);
     return fmaxf(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
   }
-  return fmaxf(max3(__uint_as_float(v.x), __uint_as_float(v.y), __uint_as_float(v.z)), __uint_as_float(v.w));
+  float m = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < N; ++j)
+    m = fmaxf(fmaxf(max3(__uint_as_float(v[j].x), __uint_as_float(v[j].y), __uint_as_float(v[j].z)), __uint_as_float(v[j].w)), m);
+  return m;
 }
 
 // Packed single precision: two fp32 values in one 64-bit register, one instruction for both
@@ -350,19 +361,53 @@ static __global__ void __launch_bounds__(256)
   row_cf[n] = cf > 0.f ? cf : 0.f;
 }
 
-// Zeros for the rows the on-chip kernel does not differentiate, one CTA per row, so that the
-// on-chip kernel only ever sees rows it works on.  Launched AFTER the on-chip kernel with
-// programmatic stream serialisation: the on-chip kernel lets its dependents go at once, so
-// these CTAs run next to it on the SMs its clusters leave free (13 of 148 with clusters of
-// nine) and, whatever is left when it ends, on all SMs.  The two kernels write disjoint rows.
-// CTA 0 ends by waiting for the on-chip kernel, so that this grid -- which is what the next
-// launch in the stream waits for -- is not complete before the on-chip kernel is.
+// Zeros for the rows the on-chip kernel does not differentiate, so that the on-chip kernel only
+// ever sees rows it works on.  A CTA is one warp with a 48 KB buffer of zeros in shared memory;
+// one lane writes a row with bulk asynchronous copies shared -> global, which take no further
+// instructions.  Launched AFTER the on-chip kernel with programmatic stream serialisation: the
+// on-chip kernel lets its dependents go at once, so these CTAs run on the SMs its clusters leave
+// free (13 of 148 with clusters of nine) while it works and on all SMs once it has ended.  The
+// buffer is larger than what an SM's shared-memory configuration leaves beside an on-chip CTA
+// (the configurations are at most 36 KB apart), on purpose: zero-fill CTAs that shared an SM with
+// on-chip CTAs slowed those down by more than they gained (measured with 16 KB buffers; 32, 40
+// and 48 KB are within 1 % of each other, 48 first).  The
+// two kernels write disjoint rows.  CTA 0 ends by waiting for the on-chip kernel, so that this
+// grid -- which is what the next launch in the stream waits for -- is not complete before the
+// on-chip kernel is.
+constexpr uint32_t kZeroBufBytes = 49152;
 template <int DT>
-__global__ void __launch_bounds__(256) zero_rows_kernel(ChunkDev c, const float *row_cf, void *dlogits) {
+__global__ void __launch_bounds__(32) zero_rows_kernel(ChunkDev c, const float *row_cf, void *dlogits) {
   using E = Elem<DT>;
-  for (int64_t n = blockIdx.x; n < c.n_rows; n += gridDim.x)
-    if (!(row_cf[n] > 0.f))
-      zero_fill_row<DT, 256>(reinterpret_cast<char *>(dlogits) + n * c.stride * E::kBytes, c.vocab);
+  extern __shared__ __align__(128) unsigned char zero_buf[];
+  const int lane = threadIdx.x;
+  const int64_t pitch = c.stride * E::kBytes;
+  const int64_t bulk_bytes = (c.vocab * E::kBytes) & ~int64_t(15);  // the rest of a row (< 16 bytes) by plain stores
+  bool ready = false;
+  for (int64_t n = blockIdx.x; n < c.n_rows; n += gridDim.x) {
+    if (row_cf[n] > 0.f) continue;
+    if (!ready) {
+      for (uint32_t i = lane * 16u; i < kZeroBufBytes; i += 32u * 16u)
+        *reinterpret_cast<uint4 *>(zero_buf + i) = make_uint4(0u, 0u, 0u, 0u);
+      // the zeros were written through the generic proxy; the copies read them through the async proxy
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      ready = true;
+    }
+    char *orow = reinterpret_cast<char *>(dlogits) + n * pitch;
+    if (lane == 0) {
+      const uint32_t src = smem_u32(zero_buf);
+      for (int64_t off = 0; off < bulk_bytes; off += kZeroBufBytes) {
+        const uint32_t bytes = (uint32_t)min((int64_t)kZeroBufBytes, bulk_bytes - off);
+        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(orow + off), "r"(src), "r"(bytes)
+                     : "memory");
+      }
+      asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    }
+    const int64_t tail = bulk_bytes / E::kBytes + lane;
+    if (tail < c.vocab) E::store1(orow, tail, 0.f);
+  }
+  // the buffer must outlive the copies that read it; they are this thread's own and always complete
+  if (ready && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   if (blockIdx.x == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
@@ -384,6 +429,7 @@ struct ClusterShared {
   unsigned long long free_t_bar[kTeacherBufs];  // teacher slice no longer needed (one arrival per compute warp)
   unsigned long long red_bar[2];             // [row parity] warp partials written (one arrival per compute warp)
   unsigned long long grad_bar[2];            // [row parity] rec ready (1 arrival)
+  uint4 no_logit;                            // filler for register slots without a vector
   unsigned long long xchg_bar[2];            // [row parity] partials of all CTAs here (1 arrival + bytes)
   float4 partial4[2][kMaxClusterSize];       // [row parity][source CTA rank] {ms, zs, as, mt}, written by peers
   float partial_zt[2][kMaxClusterSize];      // [row parity][source CTA rank] zt
@@ -391,7 +437,6 @@ struct ClusterShared {
   RowAcc warp_scratch[2][kFusedMaxWarps];    // [row parity][compute warp]
   RowRec rec[2];                             // [row parity]
   long long first_rows[2];                   // the cluster's first two differentiated rows (or -1)
-  uint4 no_logit;                            // filler for register slots without a vector
   int failed;                                // a bounded wait ran out somewhere in this CTA
 };
 
@@ -669,11 +714,8 @@ __global__ void __launch_bounds__(W * 32 + 32, 1) fused_cluster_kernel(FusedArgs
           X[j] = lds128(j < nv ? s_base + voff[j] : no_logit);
           T[j] = lds128(j < nv ? t_base + voff[j] : no_logit);
         }
-#pragma unroll
-        for (int j = 0; j < NV; ++j) {
-          acc.ms = fmaxf(acc.ms, vec_max<DT>(X[j]));
-          acc.mt = fmaxf(acc.mt, vec_max<DT>(T[j]));
-        }
+        acc.ms = vecs_max<DT, NV>(X);
+        acc.mt = vecs_max<DT, NV>(T);
         if (has_tail) {
           x_tail_s = E::load1(reinterpret_cast<const char *>(c.student) + cur * row_bytes, tail_idx);
           x_tail_t = E::load1(reinterpret_cast<const char *>(c.teacher) + cur * row_bytes, tail_idx);
@@ -689,7 +731,17 @@ __global__ void __launch_bounds__(W * 32 + 32, 1) fused_cluster_kernel(FusedArgs
         // goes back (the warp-wide maximum has also brought the lanes together)
         if (lane == 0) mbar_arrive_after(smem_u32(&sh.free_s_bar[sb]), acc.ms);
         {
-          const f32x2 ms2 = pack2(acc.ms, acc.ms), mt2 = pack2(acc.mt, acc.mt), l2 = pack2(kLog2e, kLog2e);
+          // Exponent (x - max) * log2(e) in one fused multiply-add, x * log2(e) - c with c =
+          // fl(max * log2(e)).  The product is exact inside the fma, so the result is off by the
+          // rounding of c alone, c_lo = max * log2(e) - c, which the next fma gives exactly and
+          // which is the same for every element of the warp: the sums come out scaled by
+          // 2^c_lo and are put right afterwards (|c_lo| < 1e-4, so 2^-c_lo = 1 - c_lo ln 2 to
+          // 1e-9).  The accuracy does not depend on the size of the logits.
+          // (a warp with nothing but filler slots: its maximum is kept away from overflow in c)
+          const float ms_f = fmaxf(acc.ms, -2e38f), mt_f = fmaxf(acc.mt, -2e38f);
+          const float cs = ms_f * kLog2e, ct = mt_f * kLog2e;
+          const float cs_lo = fmaf(ms_f, kLog2e, -cs), ct_lo = fmaf(mt_f, kLog2e, -ct);
+          const f32x2 cs2 = pack2(-cs, -cs), ct2 = pack2(-ct, -ct), l2 = pack2(kLog2e, kLog2e);
           f32x2 zs2 = pack2(0.f, 0.f), as2 = zs2, zt2 = zs2;  // student and teacher sums take the same steps
 #pragma unroll
           for (int j = 0; j < NV; ++j) {
@@ -698,20 +750,20 @@ __global__ void __launch_bounds__(W * 32 + 32, 1) fused_cluster_kernel(FusedArgs
             PP::get(T[j], t2);
 #pragma unroll
             for (int q = 0; q < PP::kPairs; ++q) {
-              // (x - max) * log2(e): the difference first, so the result does not degrade with the size of the logits
-              const f32x2 es = ex2_2(mul2(sub2(s2[q], ms2), l2)), et = ex2_2(mul2(sub2(t2[q], mt2), l2));
+              const f32x2 es = ex2_2(fma2(s2[q], l2, cs2)), et = ex2_2(fma2(t2[q], l2, ct2));
               zs2 = add2(zs2, es);
               as2 = fma2(es, sub2(s2[q], t2[q]), as2);
               zt2 = add2(zt2, et);
             }
           }
+          const float fix_s = -cs_lo * kLn2, fix_t = -ct_lo * kLn2;
           float lo, hi;
           unpack2(zs2, lo, hi);
-          acc.zs = lo + hi;
+          acc.zs = fmaf(lo + hi, fix_s, lo + hi);
           unpack2(as2, lo, hi);
-          acc.as = lo + hi;
+          acc.as = fmaf(lo + hi, fix_s, lo + hi);
           unpack2(zt2, lo, hi);
-          acc.zt = lo + hi;
+          acc.zt = fmaf(lo + hi, fix_t, lo + hi);
         }
         if (has_tail) {
           const float e = ex2((x_tail_s - acc.ms) * kLog2e);

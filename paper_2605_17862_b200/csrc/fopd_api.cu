@@ -58,6 +58,8 @@ static bool fused_shape_for(int64_t slice, int *nv, int *warps) {
 }
 
 static int set_fused_attributes(const void *kernel, int C, size_t smem) {
+  // (all of the SM's configurable memory as shared memory: the kernel hardly uses the L1, and the
+  // small CTAs that write the zero rows beside it need room for their buffers)
   if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
       cudaFuncSetAttribute(kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, C > 8 ? 1 : 0) != cudaSuccess) {
     (void)cudaGetLastError();
@@ -222,8 +224,9 @@ int launch_fused(const fopd_chunk *chunk, int32_t B, const float *coef, float la
   zattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   zattr[0].val.programmaticStreamSerializationAllowed = 1;
   cudaLaunchConfig_t zcfg = cudaLaunchConfig_t{};
-  zcfg.blockDim = dim3(256);
+  zcfg.blockDim = dim3(32);
   zcfg.gridDim = dim3(row_grid(chunk->n_rows));
+  zcfg.dynamicSmemBytes = kZeroBufBytes;
   zcfg.stream = st;
   zcfg.attrs = zattr;
   zcfg.numAttrs = 1;
