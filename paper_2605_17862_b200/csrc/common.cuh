@@ -116,34 +116,6 @@ struct RowAcc {
     ms = mt = kNegBig;
     zs = as = zt = 0.f;
   }
-  // Fold N (s, t) pairs in; the maxima move only when a vector beats them.
-  template <int N>
-  __device__ __forceinline__ void add(const float (&s)[N], const float (&t)[N]) {
-    const float vs = max_of<N>(s), vt = max_of<N>(t);
-    if (vs > ms) {
-      const float r = ex2((ms - vs) * kLog2e);
-      zs *= r;
-      as *= r;
-      ms = vs;
-    }
-    if (vt > mt) {
-      zt *= ex2((mt - vt) * kLog2e);
-      mt = vt;
-    }
-    // (x - max) * log2(e), not x * log2(e) - max * log2(e) in one fused multiply-add: the
-    // difference is (nearly) exact, so the result does not degrade with the size of the logits
-#pragma unroll
-    for (int i = 0; i < N; ++i) {
-      const float es = ex2((s[i] - ms) * kLog2e);
-      zs += es;
-      as = fmaf(es, s[i] - t[i], as);
-      zt += ex2((t[i] - mt) * kLog2e);
-    }
-  }
-  __device__ __forceinline__ void add1(float s, float t) {
-    const float a[1] = {s}, b[1] = {t};
-    add<1>(a, b);
-  }
   // Merge another partial (order of the two operands does not change the
   // maxima; the sums are combined lower-index first by the callers).
   __device__ __forceinline__ void merge(const RowAcc &o) {
@@ -157,6 +129,64 @@ struct RowAcc {
     const float ta = ex2((mt - Mt) * kLog2e), tb = ex2((o.mt - Mt) * kLog2e);
     zt = __fmaf_rn(zt, ta, __fmul_rn(o.zt, tb));
     mt = Mt;
+  }
+};
+
+// The accumulators of one thread while it sweeps its part of a row.  The exponent
+// (x - max) * log2(e) is formed by one fused multiply-add, x * log2(e) - c with c =
+// fl(max * log2(e)): the product is exact inside the fma, so the result differs from the
+// exponent wanted only by the rounding of c, c_lo = max * log2(e) - c, which is the same for
+// every element.  The sums therefore come out scaled by 2^c_lo exactly as they would with the
+// difference taken first, and settle() takes the factor out (c_lo is given exactly by one more
+// fma; |c_lo| < 1e-4, so 2^-c_lo = 1 - c_lo ln 2 to 1e-9).  The accuracy does not depend on the
+// size of the logits.  When a maximum moves, the sums go from scale 2^-c_old to 2^-c_new by the
+// factor 2^(c_old - c_new).  Student and teacher sums take the same steps, so a teacher equal
+// to the student gives equal sums bit for bit.
+struct RowSweep {
+  float ms, cs, zs, as, mt, ct, zt;
+  __device__ __forceinline__ void init() {
+    ms = mt = cs = ct = kNegBig;
+    zs = as = zt = 0.f;
+  }
+  // Fold N (s, t) pairs in; the maxima move only when a vector beats them.
+  template <int N>
+  __device__ __forceinline__ void add(const float (&s)[N], const float (&t)[N]) {
+    const float vs = max_of<N>(s), vt = max_of<N>(t);
+    if (vs > ms) {
+      const float cn = vs * kLog2e, r = ex2(cs - cn);
+      zs *= r;
+      as *= r;
+      ms = vs;
+      cs = cn;
+    }
+    if (vt > mt) {
+      const float cn = vt * kLog2e;
+      zt *= ex2(ct - cn);
+      mt = vt;
+      ct = cn;
+    }
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+      const float es = ex2(fmaf(s[i], kLog2e, -cs));
+      zs += es;
+      as = fmaf(es, s[i] - t[i], as);
+      zt += ex2(fmaf(t[i], kLog2e, -ct));
+    }
+  }
+  __device__ __forceinline__ void add1(float s, float t) {
+    const float a[1] = {s}, b[1] = {t};
+    add<1>(a, b);
+  }
+  // The thread's partial on the scale of its own maxima, ready to be merged.
+  __device__ __forceinline__ RowAcc settle() const {
+    const float fs = -fmaf(ms, kLog2e, -cs) * kLn2, ft = -fmaf(mt, kLog2e, -ct) * kLn2;
+    RowAcc r;
+    r.ms = ms;
+    r.zs = __fmaf_rn(zs, fs, zs);
+    r.as = __fmaf_rn(as, fs, as);
+    r.mt = mt;
+    r.zt = __fmaf_rn(zt, ft, zt);
+    return r;
   }
 };
 

@@ -92,7 +92,7 @@ template <int DT, int kThreads>
 __device__ __forceinline__ RowAcc sweep_row_global(const void *srow, const void *trow, int64_t V) {
   using E = Elem<DT>;
   constexpr int P = E::kPerVec;
-  RowAcc acc;
+  RowSweep acc;
   acc.init();
   const int64_t nvec = V / P;
   const uint4 *s4 = reinterpret_cast<const uint4 *>(srow);
@@ -121,7 +121,7 @@ __device__ __forceinline__ RowAcc sweep_row_global(const void *srow, const void 
   }
   const int64_t tail = nvec * P + threadIdx.x;
   if (tail < V) acc.add1(E::load1(srow, tail), E::load1(trow, tail));
-  return acc;
+  return acc.settle();
 }
 
 // a1-a4: statistics sweep.  grid = rows (any grid works), block = kThreads.
