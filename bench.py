@@ -45,7 +45,8 @@ FALLBACK_HBM_GBS = 6650.0
 # L2, a few GB on the device); the traffic of a row does not depend on how many rows there are, so
 # the ratio scales to a full launch by the rows processed.  A kernel that has changed since its
 # counters were taken is taken out of this table (traffic: null).
-NCU_TRAFFIC_RATIO = {"grad_stream_kernel": 0.990, "token_stats_kernel": 1.000}
+NCU_TRAFFIC_RATIO = {"grad_stream_kernel": 0.989, "token_stats_kernel": 1.001, "fused_cluster_kernel": 0.990,
+                     "grad_sampled_kernel": 0.979}
 
 def parse_args():
     ap = argparse.ArgumentParser()
