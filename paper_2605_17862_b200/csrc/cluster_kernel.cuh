@@ -84,17 +84,11 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 // Arrival with release semantics (the default): what the arriving thread read or wrote before
-// it is ordered before whatever the thread that sees the phase complete does next.
+// it is ordered before whatever the thread that sees the phase complete does next.  Slice
+// buffers are handed back with it (the warp's reads of the buffer, then the arrival; the control
+// warp starts the copy that overwrites the buffer only after it has seen the phase complete).
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-// Arrival that orders nothing by itself.  Used to hand a slice buffer back: `after` is a value
-// computed from everything the thread loaded out of the buffer, so the instruction cannot issue
-// before those loads have returned their data, and a load that has returned is not affected by
-// the copy that overwrites the buffer afterwards.  (A releasing arrival would also wait for the
-// thread's outstanding global stores, which have nothing to do with the buffer.)
-__device__ __forceinline__ void mbar_arrive_after(uint32_t bar, float after) {
-  asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];" ::"r"(bar), "f"(after) : "memory");
 }
 // Stores into another CTA's shared memory that also credit their bytes to an mbarrier of
 // that CTA: the receiver's wait on the barrier covers the data, the sender needs no fence.
@@ -731,7 +725,8 @@ __global__ void __launch_bounds__(W * 32 + 32, 1) fused_cluster_kernel(FusedArgs
         acc.mt = warp_max(acc.mt);
         // the student slice is in registers now (the maxima have looked at all of it): its buffer
         // goes back (the warp-wide maximum has also brought the lanes together)
-        if (lane == 0) mbar_arrive_after(smem_u32(&sh.free_s_bar[sb]), acc.ms);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&sh.free_s_bar[sb]));
         {
           // Exponent (x - max) * log2(e) in one fused multiply-add, x * log2(e) - c with c =
           // fl(max * log2(e)).  The product is exact inside the fma, so the result is off by the
@@ -804,7 +799,6 @@ __global__ void __launch_bounds__(W * 32 + 32, 1) fused_cluster_kernel(FusedArgs
         uint4 *o4 = reinterpret_cast<uint4 *>(orow) + v_lo + ctid;
         const bool token_here = y_owner == ctid;
         const f32x2 l2g = pack2(kLog2e, kLog2e), e2g = pack2(gr.e0, gr.e0), K2g = pack2(gr.K, gr.K);
-        float seen = 0.f;  // depends on every teacher vector read below
 #pragma unroll
         for (int j = 0; j < NV; ++j) {
           f32x2 s2[PP::kPairs], t2[PP::kPairs], o2[PP::kPairs];
@@ -828,12 +822,11 @@ __global__ void __launch_bounds__(W * 32 + 32, 1) fused_cluster_kernel(FusedArgs
             }
           }
           const uint4 o = PP::put(o2);
-          seen += __uint_as_float(o.x & 0x007fffffu);
           if (j < nv) st_stream(o4 + j * kFusedCompute, o);
         }
         // the teacher slice has been read for the last time: its buffer goes back
         __syncwarp();
-        if (lane == 0) mbar_arrive_after(smem_u32(&sh.free_t_bar[tb]), seen);
+        if (lane == 0) mbar_arrive(smem_u32(&sh.free_t_bar[tb]));
         if (has_tail) {
           float o = ex2(fmaf(y_tail_s, kLog2e, gr.e0)) * ((y_tail_s - y_tail_t) - gr.K);
           if (tail_idx == gr.y) o = fmaf(ex2(fmaf(y_tail_s, kLog2e, gr.e0)), (y_tail_s - y_tail_t) - gr.K, gr.cg);
