@@ -372,6 +372,27 @@ def main():
         torch.cuda.synchronize()
         on_chip_ms = t_begin.elapsed_time(t_end) / args.steps
 
+    # the whole step with the fewest bytes: the measurement phase reads the student rows only
+    # (all the freshness needs), the loss phase runs without cached statistics
+    student_step = None
+    if cached and not args.no_on_chip:
+        ev_s = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        for it in range(3 + args.steps):
+            if it == 3:
+                torch.cuda.synchronize()
+                t_begin.record()
+            buf.reset()
+            if it == 3 + args.steps - 1: ev_s[0].record()
+            pl.measure_student(chunks, buf, None)
+            if it == 3 + args.steps - 1: ev_s[1].record()
+            pl.freshness(buf, tau, H, None, p)
+            pl.optimise(chunks, dlogits, buf, p, None, use_row_ws=False)
+        t_end.record()
+        torch.cuda.synchronize()
+        assert fb.fopd_check_status(buf.status) == 0
+        student_step = {"ms_per_batch": t_begin.elapsed_time(t_end) / args.steps,
+                        "student_stats_ms_last_step": ev_s[0].elapsed_time(ev_s[1]), "loss": float(buf.loss.cpu()[0])}
+
     # the sampled-token form of the token loss (importance-weighted reverse KL on the stored token):
     # its own measurement phase for the row statistics and weights, then the timed loss forward +
     # backward, which reads only the student row of a differentiated row
@@ -464,6 +485,11 @@ def main():
             "loss_fwd_bwd_cached" if cached else "loss_fwd_bwd_standalone": dict(
                 figure(grad_ms, grad_bytes, active_rows), kernel=grad_kernel,
                 bytes="3 V e per differentiated row, V e per other row"),
+            "whole_step_student_statistics": None if student_step is None else dict(
+                figure(student_step["ms_per_batch"], stats_bytes / 2 + grad_bytes, aligned),
+                student_stats_ms=student_step["student_stats_ms_last_step"], loss=student_step["loss"],
+                calls="fopd_token_stats_student, fopd_sample_freshness, fopd_loss_fwd_bwd(row_ws = NULL), fopd_loss_finalize",
+                bytes="V e per aligned row, then 3 V e per differentiated row (V e per other row): 4 V e in all"),
             "loss_fwd_bwd_on_chip": None if on_chip_ms is None else dict(
                 figure(on_chip_ms, grad_bytes, active_rows), kernel=on_chip_kernel, plan=plan),
             "loss_fwd_bwd_sampled_token_form": sampled,

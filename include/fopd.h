@@ -73,7 +73,7 @@
 extern "C" {
 #endif
 
-#define FOPD_VERSION 200
+#define FOPD_VERSION 201
 
 typedef enum { FOPD_BF16 = 0, FOPD_F32 = 1 } fopd_dtype;
 
@@ -178,6 +178,25 @@ typedef struct {
 int fopd_token_stats(const fopd_chunk *chunk /* HOST */, int32_t B, float *lp_s,
                      float *lp_t, float *kl, float *ratio, float *row_ws,
                      double *acc, int32_t *status, void *stream);
+
+/*
+ * The student's half of fopd_token_stats: what the measurement loop of Algorithm 1
+ * needs and no more.  The rollout drift (Eq. 10), the freshness score (Eq. 11) and
+ * the gate (Eq. 13) depend on the student's and the behaviour policy's
+ * log-probabilities of the stored tokens only, so this call reads the student rows
+ * alone (V * e bytes per aligned row instead of 2 * V * e) and never touches
+ * chunk->teacher, which may be NULL.  acc gets the count, the k3 sum and the row
+ * count; its FOPD_ACC_KL column is left as it is, so fopd_sample_freshness reports
+ * l_distill = 0 for such a batch.  The loss phase then runs fopd_loss_fwd_bwd with
+ * row_ws = NULL (this call leaves no row statistics behind): 4 * V * e bytes per
+ * differentiated token for the whole step instead of 5 * V * e.
+ *
+ *   lp_s, ratio   [n_rows] fp32 outputs, either may be NULL; exactly 0 for rows
+ *                 with mask = 0 or a bad id.
+ *   acc, status, stream, errors, the temporary: as for fopd_token_stats.
+ */
+int fopd_token_stats_student(const fopd_chunk *chunk /* HOST */, int32_t B, float *lp_s,
+                             float *ratio, double *acc, int32_t *status, void *stream);
 
 /*
  * fopd_token_stats for callers that must not allocate device memory.  (The

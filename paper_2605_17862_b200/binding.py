@@ -23,6 +23,7 @@ EXPORTS = (
     "fopd_token_stats_static", "fopd_loss_fwd_bwd_plan", "fopd_row_divergence", "fopd_supervision_drift",
     "fopd_refresh_decision", "fopd_shard_stats", "fopd_shard_merge", "fopd_shard_loss_fwd_bwd",
     "fopd_loss_fwd_bwd_set_plan", "fopd_release_device_memory", "fopd_selftest_bounded_wait",
+    "fopd_token_stats_student",
 )
 
 
@@ -69,6 +70,7 @@ def lib() -> ctypes.CDLL:
         L.fopd_strerror.restype = ctypes.c_char_p
         L.fopd_strerror.argtypes = [ctypes.c_int]
         L.fopd_token_stats.argtypes = [ctypes.POINTER(fopd_chunk), i32, vp, vp, vp, vp, vp, vp, vp, vp]
+        L.fopd_token_stats_student.argtypes = [ctypes.POINTER(fopd_chunk), i32, vp, vp, vp, vp, vp]
         L.fopd_token_stats_static.argtypes = [ctypes.POINTER(fopd_chunk), i32, vp, vp, vp, vp, vp, vp, vp]
         L.fopd_sample_freshness.argtypes = [vp, vp, vp, vp, i32, fopd_params, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         L.fopd_loss_fwd_bwd.argtypes = [ctypes.POINTER(fopd_chunk), i32, vp, vp, fopd_params, vp, vp, vp, vp]
@@ -127,7 +129,7 @@ def params(alpha=1.0, beta=1.0, xi=0.15, lam=0.1) -> fopd_params:
 class Chunk:
     """Device tensors of one chunk of token rows (see ``fopd_chunk`` in fopd.h)."""
     student: torch.Tensor  # [n, V] (row pitch = student.stride(0)), bf16 or fp32
-    teacher: torch.Tensor
+    teacher: torch.Tensor | None  # None only for fopd_token_stats_student
     behav_logprob: torch.Tensor  # [n] fp32
     tokens: torch.Tensor  # [n] int32
     mask: torch.Tensor  # [n] uint8
@@ -137,15 +139,15 @@ class Chunk:
 
     def c_struct(self) -> fopd_chunk:
         S, T = self.student, self.teacher
-        assert S.dtype == T.dtype and S.dtype in (torch.bfloat16, torch.float32)
-        assert S.dim() == 2 and S.shape == T.shape and S.stride() == T.stride() and S.stride(1) == 1
+        assert S.dtype in (torch.bfloat16, torch.float32) and S.dim() == 2 and S.stride(1) == 1
+        assert T is None or (S.dtype == T.dtype and S.shape == T.shape and S.stride() == T.stride())
         assert self.behav_logprob.dtype == torch.float32 and self.tokens.dtype == torch.int32
         assert self.mask.dtype == torch.uint8 and self.sample_id.dtype == torch.int32
         n = S.shape[0]
         for t in (self.behav_logprob, self.tokens, self.mask, self.sample_id):
             assert t.is_contiguous() and t.numel() == n and t.device == S.device
         return fopd_chunk(
-            S.data_ptr(), T.data_ptr(), self.behav_logprob.data_ptr(), self.tokens.data_ptr(),
+            S.data_ptr(), None if T is None else T.data_ptr(), self.behav_logprob.data_ptr(), self.tokens.data_ptr(),
             self.mask.data_ptr(), self.sample_id.data_ptr(), n, self.vocab or S.shape[1],
             S.stride(0) if n > 1 else max(S.stride(0), S.shape[1]),
             FOPD_BF16 if S.dtype == torch.bfloat16 else FOPD_F32, int(self.loss_kind),
@@ -158,6 +160,15 @@ def fopd_token_stats(chunk: Chunk, B: int, acc, *, lp_s=None, lp_t=None, kl=None
     _check(lib().fopd_token_stats(ctypes.byref(c), B, _ptr(lp_s), _ptr(lp_t), _ptr(kl), _ptr(ratio),
                                   _ptr(row_ws), _ptr(acc), _ptr(status), _stream(stream)),
            "fopd_token_stats")
+
+
+def fopd_token_stats_student(chunk: Chunk, B: int, acc, *, lp_s=None, ratio=None, status=None, stream=None):
+    """The student's half of fopd_token_stats (chunk.teacher may be None): enough for
+    fopd_sample_freshness; the loss call that follows gets no row_ws."""
+    c = chunk.c_struct()
+    _check(lib().fopd_token_stats_student(ctypes.byref(c), B, _ptr(lp_s), _ptr(ratio), _ptr(acc), _ptr(status),
+                                          _stream(stream)),
+           "fopd_token_stats_student")
 
 
 STATIC_MAX_ROWS = 65536

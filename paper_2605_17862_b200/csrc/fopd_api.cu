@@ -286,6 +286,41 @@ int fopd_token_stats(const fopd_chunk *chunk, int32_t B, float *lp_s, float *lp_
   return rc;
 }
 
+int fopd_token_stats_student(const fopd_chunk *chunk, int32_t B, float *lp_s, float *ratio, double *acc,
+                             int32_t *status, void *stream) {
+  int rc = check_chunk(chunk, B, false);
+  if (rc != FOPD_OK) return rc;
+  if (!acc) return FOPD_ERR_NULL;
+  if (chunk->n_rows == 0) return FOPD_OK;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t bb = (bounds_bytes(B) + 255) & ~size_t(255);
+  char *tmp = nullptr;
+  if ((rc = scratch_alloc(reinterpret_cast<void **>(&tmp), bb + (size_t)chunk->n_rows * 4 * sizeof(float), st)) != FOPD_OK)
+    return rc;
+  unsigned long long *bounds = reinterpret_cast<unsigned long long *>(tmp);
+  float *ws = reinterpret_cast<float *>(tmp + bb);
+  const ChunkDev d = to_dev(chunk);
+  const unsigned grid = row_grid(chunk->n_rows);
+  const bool short_row = chunk->vocab / (chunk->dtype == FOPD_BF16 ? 8 : 4) < kShortRowVecs;
+#define FOPD_LAUNCH_STUDENT(DT, T) token_stats_student_kernel<DT, T><<<grid, T, 0, st>>>(d, B, lp_s, ratio, ws, status)
+  if (chunk->dtype == FOPD_BF16) {
+    if (short_row) FOPD_LAUNCH_STUDENT(FOPD_BF16, kStatsThreadsShortRow);
+    else FOPD_LAUNCH_STUDENT(FOPD_BF16, kStatsThreads);
+  } else {
+    if (short_row) FOPD_LAUNCH_STUDENT(FOPD_F32, kStatsThreadsShortRow);
+    else FOPD_LAUNCH_STUDENT(FOPD_F32, kStatsThreads);
+  }
+#undef FOPD_LAUNCH_STUDENT
+  rc = launch_ok();
+  if (rc == FOPD_OK) rc = launch_sample_bounds(chunk->sample_id, chunk->n_rows, B, bounds, st);
+  if (rc == FOPD_OK) {
+    segment_reduce_kernel<<<B, kSegThreads, 0, st>>>(d, B, ws, nullptr, 0, bounds_or_null(bounds, B), acc);
+    rc = launch_ok();
+  }
+  if (cudaFreeAsync(tmp, st) != cudaSuccess) rc = FOPD_ERR_CUDA;
+  return rc;
+}
+
 int fopd_sample_freshness(const double *acc, const int32_t *staleness, const int32_t *seq_len,
                           const float *d_sup, int32_t B, fopd_params p, float *f, float *w,
                           float *d_roll, float *l_distill, float *m_align, float *coef,

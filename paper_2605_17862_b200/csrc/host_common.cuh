@@ -11,17 +11,17 @@ namespace fopd {
 
 static inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-static inline int check_chunk(const fopd_chunk *c, int32_t B) {
+static inline int check_chunk(const fopd_chunk *c, int32_t B, bool needs_teacher = true) {
   if (!c) return FOPD_ERR_NULL;
   if (c->dtype != FOPD_BF16 && c->dtype != FOPD_F32) return FOPD_ERR_DTYPE;
   if (c->loss_kind != FOPD_LOSS_FULL_KL && c->loss_kind != FOPD_LOSS_SAMPLED_KL) return FOPD_ERR_KIND;
   if (c->n_rows < 0 || c->vocab <= 0 || c->row_stride < c->vocab || B <= 0) return FOPD_ERR_SIZE;
   if (c->vocab > (int64_t)1 << 30 || c->n_rows > (int64_t)1 << 40) return FOPD_ERR_SIZE;
   if (c->n_rows == 0) return FOPD_OK;
-  if (!c->student || !c->teacher || !c->behav_logprob || !c->tokens || !c->mask || !c->sample_id)
+  if (!c->student || (needs_teacher && !c->teacher) || !c->behav_logprob || !c->tokens || !c->mask || !c->sample_id)
     return FOPD_ERR_NULL;
   const int64_t esz = c->dtype == FOPD_BF16 ? 2 : 4;
-  if (!aligned16(c->student) || !aligned16(c->teacher) || (c->row_stride * esz) % 16 != 0)
+  if (!aligned16(c->student) || (needs_teacher && !aligned16(c->teacher)) || (c->row_stride * esz) % 16 != 0)
     return FOPD_ERR_ALIGN;
   return FOPD_OK;
 }

@@ -154,6 +154,88 @@ __global__ void __launch_bounds__(kThreads, 1024 / kThreads)
   }
 }
 
+// Student-only statistics sweep: what the first loop of Algorithm 1 needs (Eq. 10, Eq. 11: the
+// rollout drift and the freshness depend on the student's and the behaviour policy's
+// log-probabilities of the stored tokens alone).  One read of the student row, one ex2 per logit;
+// the exponent is formed as in RowSweep.  row_ws gets {lse_s, 0, 0, d}: enough for the
+// per-sample sums, not for the gradient sweep.
+template <int DT, int kThreads>
+__device__ __forceinline__ RowAcc sweep_row_student(const void *srow, int64_t V) {
+  using E = Elem<DT>;
+  constexpr int P = E::kPerVec;
+  float ms = kNegBig, cs = kNegBig, zs = 0.f;
+  auto add = [&](const float *s, int n) {
+    float vs = s[0];
+    for (int i = 1; i < n; ++i) vs = fmaxf(vs, s[i]);
+    if (vs > ms) {
+      const float cn = vs * kLog2e;
+      zs *= ex2(cs - cn);
+      ms = vs;
+      cs = cn;
+    }
+    for (int i = 0; i < n; ++i) zs += ex2(fmaf(s[i], kLog2e, -cs));
+  };
+  const int64_t nvec = V / P;
+  const uint4 *s4 = reinterpret_cast<const uint4 *>(srow);
+  int64_t i = threadIdx.x;
+  constexpr int kU = 2 * kUnroll;  // half the loads per vector of the two-row sweep: twice the vectors in flight
+  for (; i + (kU - 1) * kThreads < nvec; i += kU * kThreads) {
+    uint4 a[kU];
+#pragma unroll
+    for (int u = 0; u < kU; ++u) a[u] = ld_stream(s4 + i + u * kThreads);
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      float s[P];
+      E::unpack(a[u], s);
+      add(s, P);
+    }
+  }
+  for (; i < nvec; i += kThreads) {
+    float s[P];
+    E::unpack(ld_stream(s4 + i), s);
+    add(s, P);
+  }
+  const int64_t tail = nvec * P + threadIdx.x;
+  if (tail < V) {
+    const float s1 = E::load1(srow, tail);
+    add(&s1, 1);
+  }
+  RowAcc r;
+  r.init();
+  r.ms = ms;
+  r.zs = __fmaf_rn(zs, -fmaf(ms, kLog2e, -cs) * kLn2, zs);  // the rounding of the scaled maximum, taken out
+  return r;
+}
+
+template <int DT, int kThreads>
+__global__ void __launch_bounds__(kThreads, 1024 / kThreads)
+    token_stats_student_kernel(ChunkDev c, int32_t B, float *lp_s, float *ratio, float *row_ws, int32_t *status) {
+  using E = Elem<DT>;
+  __shared__ RowAcc scratch[2][kThreads / 32];  // alternating per row: no barrier after the row's finish
+  int par = 0;
+  for (int64_t n = blockIdx.x; n < c.n_rows; n += gridDim.x) {
+    if (!row_is_aligned(c, n, B, status, threadIdx.x == 0)) {
+      if (threadIdx.x == 0) zero_row_outputs(n, lp_s, nullptr, nullptr, ratio, row_ws);
+      continue;
+    }
+    float sy = 0.f, b = 0.f;
+    if (threadIdx.x == 0) {
+      sy = E::load1(c.student, n * c.stride + c.tokens[n]);
+      b = c.behav[n];
+    }
+    RowAcc acc = sweep_row_student<DT, kThreads>(reinterpret_cast<const char *>(c.student) + n * c.stride * E::kBytes, c.vocab);
+    acc = block_reduce<kThreads>(acc, scratch[par]);
+    if (threadIdx.x == 0) {
+      const float gs = logf(acc.zs);
+      const float lps = (sy - acc.ms) - gs, d = lps - b;
+      if (lp_s) lp_s[n] = lps;
+      if (ratio) ratio[n] = expf(d);
+      reinterpret_cast<float4 *>(row_ws)[n] = make_float4(acc.ms + gs, 0.f, 0.f, d);
+    }
+    par ^= 1;
+  }
+}
+
 // Per-row constants of the gradient sweep (see fopd_loss_fwd_bwd):
 //   dS_v = cp_v * ((s_v - t_v) - K) + [v == y] * cg
 //   cp_v = coef * p_s(v) = 2^(s_v*log2e + e0),  e0 = log2(coef) - lse_s*log2e

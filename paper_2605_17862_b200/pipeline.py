@@ -72,6 +72,17 @@ def measure(chunks, buf: BatchBuffers, rows=None, *, keep_row_ws=True, stream=No
             status=buf.status, stream=stream)
 
 
+def measure_student(chunks, buf: BatchBuffers, rows=None, *, stream=None):
+    """Measurement phase from the student rows alone (fopd_token_stats_student): all that the
+    freshness score needs.  The chunks' teacher rows are not read (and may be absent)."""
+    for j, ch in enumerate(chunks):
+        r = rows[j] if rows is not None else None
+        student_view = fb.Chunk(ch.student, None, ch.behav_logprob, ch.tokens, ch.mask, ch.sample_id, ch.vocab,
+                                ch.loss_kind)
+        fb.fopd_token_stats_student(student_view, buf.B, buf.acc, lp_s=r.lp_s if r else None,
+                                    ratio=r.ratio if r else None, status=buf.status, stream=stream)
+
+
 def freshness(buf: BatchBuffers, tau, H, d_sup, p, stream=None):
     fb.fopd_sample_freshness(buf.acc, tau, H, d_sup, buf.B, p, coef=buf.coef, f=buf.f, w=buf.w,
                              d_roll=buf.d_roll, l_distill=buf.l_distill, m_align=buf.m_align,
@@ -95,6 +106,16 @@ def step(chunks, dlogits, buf: BatchBuffers, tau, H, d_sup, p, rows=None, *, use
     measure(chunks, buf, rows, keep_row_ws=use_row_ws, stream=stream)
     freshness(buf, tau, H, d_sup, p, stream=stream)
     optimise(chunks, dlogits, buf, p, rows, use_row_ws=use_row_ws, stream=stream)
+
+
+def step_student_stats(chunks, dlogits, buf: BatchBuffers, tau, H, d_sup, p, rows=None, *, stream=None):
+    """The whole hot path with the fewest bytes: the student's statistics (V e per token), the
+    freshness, then the loss forward + backward without cached statistics (3 V e per
+    differentiated token)."""
+    buf.reset()
+    measure_student(chunks, buf, rows, stream=stream)
+    freshness(buf, tau, H, d_sup, p, stream=stream)
+    optimise(chunks, dlogits, buf, p, None, use_row_ws=False, stream=stream)
 
 
 def to_chunk(d: dict, vocab=None, loss_kind: int = fb.LOSS_FULL_KL) -> fb.Chunk:

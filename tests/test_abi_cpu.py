@@ -31,7 +31,7 @@ def test_library_exports_every_declared_symbol(lib):
     for n in names:
         assert hasattr(lib, n), f"{n} declared in fopd.h but not exported"
     assert set(names) == set(fb.EXPORTS)
-    assert fb.version() == 200
+    assert fb.version() == 201
 
 
 def test_strerror_covers_every_status(lib):
@@ -76,6 +76,14 @@ def test_more_host_checks(lib):
     assert lib.fopd_token_stats(ctypes.byref(c), 0, None, None, None, None, None, vp(0x7000), None, None) == -3
     assert lib.fopd_token_stats(ctypes.byref(c), 2, None, None, None, None, None, None, None, None) == -1
     assert lib.fopd_token_stats(ctypes.byref(c), 2, None, None, None, None, vp(0x7004), vp(0x7000), None, None) == -2
+    # the student's half of the statistics: same checks, but the teacher is not needed
+    no_teacher = _chunk(teacher=0)
+    assert lib.fopd_token_stats(ctypes.byref(no_teacher), 2, None, None, None, None, None, vp(0x7000), None, None) == -1
+    assert lib.fopd_token_stats_student(ctypes.byref(no_teacher), 2, None, None, None, None, None) == -1   # acc
+    assert lib.fopd_token_stats_student(ctypes.byref(_chunk(teacher=0, student=0)), 2, None, None, vp(0x7000), None, None) == -1
+    assert lib.fopd_token_stats_student(ctypes.byref(_chunk(teacher=0, student=0x1008)), 2, None, None, vp(0x7000), None, None) == -2
+    assert lib.fopd_token_stats_student(ctypes.byref(_chunk(teacher=0, n_rows=0)), 2, None, None, vp(0x7000), None, None) == 0
+    assert lib.fopd_token_stats_student(ctypes.byref(_chunk(teacher=0, dtype=5)), 2, None, None, vp(0x7000), None, None) == -4
     big = _chunk(n_rows=fb.STATIC_MAX_ROWS + 1)
     assert lib.fopd_token_stats_static(ctypes.byref(big), 2, None, None, None, None, vp(0x7000), None, None) == -3
     # empty chunk: nothing to do, no CUDA call

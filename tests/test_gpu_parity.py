@@ -470,3 +470,60 @@ def test_large_logit_offsets(offset, dtype):
     for use_ws in (True, False):
         out = par.compare([ch], sub.B, sub.tau, sub.H, use_row_ws=use_ws, grad_rows_per_chunk=32)
     print(offset, out)
+
+
+def test_student_only_statistics_then_loss_without_cached_statistics():
+    """Algorithm 1's first loop needs the student's and the behaviour policy's log-probabilities
+    only (Eq. 10, Eq. 11): fopd_token_stats_student must give the oracle's lp_s, ratio, counts,
+    drift sums, freshness and weights without reading the teacher, and the loss phase that
+    follows (no cached statistics) the oracle's loss and gradient."""
+    for wl, j_chunks in ((synth.coding_agent(scale=1 / 16), None), (synth.tiny(scale=1 / 4), None)):
+        chunks_dev = [synth.gen_chunk(wl, j, DEV) for j in range(wl.n_chunks)]
+        B = wl.B
+        params = par.exact(par.PARAMS)
+        p = fb.params(**params)
+        chunks = [pl.to_chunk(c) for c in chunks_dev]
+        for c in chunks_dev:  # poison the teacher for the statistics call: it must not be read
+            c["teacher_saved"] = c["teacher"].clone()
+        buf = pl.BatchBuffers(B, DEV)
+        rows = [pl.RowOutputs.alloc(c["student"].shape[0], DEV) for c in chunks_dev]
+        dlogits = [torch.full_like(c["student"], float("nan")) for c in chunks_dev]
+        tau_d = torch.as_tensor(np.asarray(wl.tau, dtype=np.int32), device=DEV)
+        H_d = torch.as_tensor(np.asarray(wl.H, dtype=np.int32), device=DEV)
+        buf.reset()
+        for c in chunks_dev:
+            c["teacher"].fill_(float("nan"))
+        pl.measure_student(chunks, buf, rows)
+        torch.cuda.synchronize()
+        for c in chunks_dev:
+            c["teacher"].copy_(c["teacher_saved"])
+        pl.freshness(buf, tau_d, H_d, None, p)
+        pl.optimise(chunks, dlogits, buf, p, None, use_row_ws=False)
+        assert fb.fopd_check_status(buf.status) == 0
+
+        hc = [par.host_chunk({k: v for k, v in c.items() if k != "teacher_saved"}) for c in chunks_dev]
+        ref = par.oracle_run(hc, B, wl.tau, wl.H, None, params)
+        for jj, st in enumerate(ref.stats):
+            valid = st.valid.astype(bool)
+            lp = rows[jj].lp_s.cpu().numpy().astype(np.float64)
+            ratio = rows[jj].ratio.cpu().numpy().astype(np.float64)
+            assert np.all(lp[~valid] == 0.0) and np.all(ratio[~valid] == 0.0)
+            assert np.abs(lp - st.lp_s)[valid].max() <= 1e-5          # observed ~1e-6; the path's bound is 1e-3
+            assert (np.abs(ratio - st.rho)[valid] / st.rho[valid]).max() <= 1e-5
+        acc = buf.acc.cpu().numpy()
+        assert np.array_equal(acc[:, 0], ref.acc[:, 0])
+        assert np.allclose(acc[:, 1], ref.acc[:, 1], rtol=par.TOL_REL, atol=1e-6 * max(1.0, ref.acc[:, 0].max()))
+        assert np.all(acc[:, 2] == 0.0)                              # no teacher, no distillation sum
+        fr = ref.fresh
+        ok = fr.f > 0
+        assert (np.abs(buf.f.cpu().numpy() - fr.f)[ok] <= par.TOL_REL * fr.f[ok]).all()
+        assert (np.abs(buf.w.cpu().numpy() - fr.w)[ok] <= par.TOL_REL * fr.f[ok]).all()
+        assert abs(float(buf.loss) - ref.loss) <= par.TOL_REL * max(abs(ref.loss), 1e-12)
+        # the gradient against the path that measured with both rows: same kernels, weights equal to ~1e-7
+        buf2, rows2, dl2, bits2 = par.gpu_run(chunks_dev, B, wl.tau, wl.H, None, params, use_row_ws=False)
+        assert bits2 == 0
+        for a, b2 in zip(dlogits, dl2):
+            a64, b64 = a.double(), b2.double()
+            assert torch.isfinite(a64).all()
+            assert ((a64 - b64).abs() <= 2 * par.out_ulp(a.dtype) * b64.abs() + 1e-12).all()
+            assert torch.equal(a64 == 0, b64 == 0)
