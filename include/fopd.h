@@ -34,6 +34,10 @@
  *     fopd_loss_finalize(...)
  *     fopd_check_status(...)
  *
+ * (fopd_token_stats_student may take the place of fopd_token_stats: the
+ * measurement phase needs the student rows only; the loss calls then get no
+ * row_ws.)
+ *
  * Memory and ownership.  Unless a parameter says HOST, every pointer is a DEVICE
  * pointer to memory the caller owns; the library keeps no pointer after a call
  * returns.  Where a call needs temporary device memory

@@ -440,7 +440,7 @@ struct FusedArgs {
   ChunkDev c;
   float lambda;
   void *dlogits;
-  const float *row_cf;  // [n_rows] from row_coef_kernel
+  const float *row_cf;  // [n_rows] from row_weight_kernel
   float *row_ws;        // [n_rows,4] out: {lse_s, lse_t, kl, d} of the differentiated rows
   int32_t *status;
   int slice_vecs;       // 16-byte vectors of a row per CTA (the last CTAs' slices may be shorter or empty)
