@@ -46,7 +46,7 @@ FALLBACK_HBM_GBS = 6650.0
 # the ratio scales to a full launch by the rows processed.  A kernel that has changed since its
 # counters were taken is taken out of this table (traffic: null).
 NCU_TRAFFIC_RATIO = {"grad_stream_kernel": 0.989, "token_stats_kernel": 1.001, "fused_cluster_kernel": 0.990,
-                     "grad_sampled_kernel": 0.979}
+                     "grad_sampled_kernel": 0.979, "token_stats_student_kernel": 1.002}
 
 def parse_args():
     ap = argparse.ArgumentParser()

@@ -50,9 +50,7 @@ namespace fopd {
 // Compute warps per CTA (W) and vectors of a row's slice a compute thread takes (NV; it holds
 // the student vectors of two rows).  Every compute thread works through NV slots whether it has
 // a vector for the last one or not, so the launcher picks the pair with the least padding.
-#define FOPD_FUSED_SHAPES(X) \
-  X(1, 19) X(2, 19) X(3, 19) X(1, 20) X(2, 20) X(3, 20) X(1, 21) X(2, 21) X(3, 21) X(1, 22) X(2, 22) X(3, 22) \
-  X(1, 23) X(2, 23) X(3, 23)
+#define FOPD_FUSED_SHAPES(X) X(1, 19) X(2, 19) X(3, 19) X(1, 21) X(2, 21) X(3, 21) X(1, 23) X(2, 23) X(3, 23)
 constexpr int kFusedMaxNV = 3, kFusedMaxWarps = 23;
 constexpr int kMaxClusterSize = 16;
 constexpr int kStudentBufs = 2, kTeacherBufs = 3;
