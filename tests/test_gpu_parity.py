@@ -477,12 +477,19 @@ def test_student_only_statistics_then_loss_without_cached_statistics():
     only (Eq. 10, Eq. 11): fopd_token_stats_student must give the oracle's lp_s, ratio, counts,
     drift sums, freshness and weights without reading the teacher, and the loss phase that
     follows (no cached statistics) the oracle's loss and gradient."""
-    for wl, j_chunks in ((synth.coding_agent(scale=1 / 16), None), (synth.tiny(scale=1 / 4), None)):
-        chunks_dev = [synth.gen_chunk(wl, j, DEV) for j in range(wl.n_chunks)]
+    # (the last case uses a vocabulary that is no multiple of the vector width: scalar tail of every row)
+    import dataclasses
+    base = synth.reasoning(scale=1 / 16)
+    ragged = dataclasses.replace(base, V=base.V - 5)
+    for wl, stride in ((synth.coding_agent(scale=1 / 16), None), (synth.tiny(scale=1 / 4), None), (ragged, base.V)):
+        drop = stride is not None
+        chunks_dev = [synth.gen_chunk(wl, j, DEV, row_stride=stride) if drop else synth.gen_chunk(wl, j, DEV)
+                      for j in range(wl.n_chunks)]
         B = wl.B
         params = par.exact(par.PARAMS)
         p = fb.params(**params)
-        chunks = [pl.to_chunk(c) for c in chunks_dev]
+        V = wl.V
+        chunks = [pl.to_chunk(c, V if drop else None) for c in chunks_dev]
         for c in chunks_dev:  # poison the teacher for the statistics call: it must not be read
             c["teacher_saved"] = c["teacher"].clone()
         buf = pl.BatchBuffers(B, DEV)
@@ -502,6 +509,10 @@ def test_student_only_statistics_then_loss_without_cached_statistics():
         assert fb.fopd_check_status(buf.status) == 0
 
         hc = [par.host_chunk({k: v for k, v in c.items() if k != "teacher_saved"}) for c in chunks_dev]
+        if drop:
+            for c in hc:
+                c["student"] = c["student"][:, :V].contiguous()
+                c["teacher"] = c["teacher"][:, :V].contiguous()
         ref = par.oracle_run(hc, B, wl.tau, wl.H, None, params)
         for jj, st in enumerate(ref.stats):
             valid = st.valid.astype(bool)
@@ -520,10 +531,11 @@ def test_student_only_statistics_then_loss_without_cached_statistics():
         assert (np.abs(buf.w.cpu().numpy() - fr.w)[ok] <= par.TOL_REL * fr.f[ok]).all()
         assert abs(float(buf.loss) - ref.loss) <= par.TOL_REL * max(abs(ref.loss), 1e-12)
         # the gradient against the path that measured with both rows: same kernels, weights equal to ~1e-7
-        buf2, rows2, dl2, bits2 = par.gpu_run(chunks_dev, B, wl.tau, wl.H, None, params, use_row_ws=False)
+        buf2, rows2, dl2, bits2 = par.gpu_run([{k: v for k, v in c.items() if k != "teacher_saved"} for c in chunks_dev], B,
+                                              wl.tau, wl.H, None, params, use_row_ws=False, vocab=V if drop else None)
         assert bits2 == 0
         for a, b2 in zip(dlogits, dl2):
-            a64, b64 = a.double(), b2.double()
+            a64, b64 = a[:, :V].double(), b2[:, :V].double()
             assert torch.isfinite(a64).all()
             assert ((a64 - b64).abs() <= 2 * par.out_ulp(a.dtype) * b64.abs() + 1e-12).all()
             assert torch.equal(a64 == 0, b64 == 0)
